@@ -1,0 +1,110 @@
+"""Pins for the oracle's decoder forward."""
+import numpy as np
+
+from oracle import oracle as O
+from paper_2608_18183_b200 import synth
+from tests import torch_restatement as TR
+
+
+def _seq(shape, n, seed):
+    rng = np.random.default_rng(seed)
+    s = rng.integers(0, shape.vocab, size=n).astype(np.int32)
+    s[0] = 0
+    return s
+
+
+def test_forward_matches_torch_restatement(tiny):
+    w, img = tiny
+    m = O.Model(w.shape, img)
+    P = TR.load(w.shape, img)
+    seq = _seq(w.shape, 23, 0)
+    got = m.forward_full(3, seq)
+    ref = TR.forward(w.shape, P, 3, seq)
+    assert np.abs(got - ref).max() < 1e-5
+    assert np.abs(ref).max() > 0.5  # the comparison is not vacuous
+
+
+def test_forward_bf16_weights_fp32_activations_matches_torch(tiny_bf16):
+    w, img = tiny_bf16
+    m = O.Model(w.shape, img, act_bf16=False)
+    P = TR.load(w.shape, img)
+    seq = _seq(w.shape, 17, 1)
+    got = m.forward_full(1, seq)
+    ref = TR.forward(w.shape, P, 1, seq)
+    assert np.abs(got - ref).max() < 2e-5
+    # with bf16 activation rounding the result moves, but stays within the bf16 budget
+    mb = O.Model(w.shape, img, act_bf16=True)
+    gb = mb.forward_full(1, seq)
+    d = np.abs(gb - ref).max()
+    assert 0 < d < 5e-2
+
+
+def test_cached_window_forward_equals_full_recompute(tiny):
+    w, img = tiny
+    m = O.Model(w.shape, img)
+    T = w.shape.T
+    seq = _seq(w.shape, T, 2)
+    full = m.forward_full(5, seq)
+    for chunks in ([T], [1] * T, [8] * 8, [5, 7, 3, 16, 1, 32]):
+        cache = m.new_cache()
+        c = 0
+        outs = []
+        for n in chunks:
+            outs.append(m.forward_window(cache, 5, seq, c, n))
+            c += n
+        got = np.concatenate(outs)
+        assert np.abs(got - full).max() < 1e-6
+
+
+def test_stale_cache_entries_are_recomputed(tiny):
+    """Entries at and after the new cursor are overwritten by the next forward: no cache repair."""
+    w, img = tiny
+    m = O.Model(w.shape, img)
+    seq = _seq(w.shape, 20, 3)
+    cache = m.new_cache()
+    m.forward_window(cache, 2, seq, 0, 6)
+    wrong = seq.copy()
+    wrong[8:14] = (wrong[8:14] + 7) % w.shape.vocab  # drafts that will be rejected
+    m.forward_window(cache, 2, wrong, 6, 8)          # writes indices 6..13, 8..13 from wrong tokens
+    got = m.forward_window(cache, 2, seq, 8, 8)      # cursor advanced to 8: recompute 8..15
+    full = m.forward_full(2, seq[:16])
+    assert np.abs(got - full[8:16]).max() < 1e-6
+
+
+def test_rope_scores_depend_on_grid_offsets_only(tiny):
+    """Shifting query and key by the same (rows, cols) on the grid leaves q.k unchanged;
+    index 0 (class token) is not rotated.  Probed through one-layer attention logits:
+    a model whose tokens all share one embedding gives position-only dependence."""
+    w, img = tiny
+    # direct check on the restated rotation: factors are unit complex numbers with angle row*w_e | col*w_e
+    rot = TR._rope_factors(w.shape, w.shape.T + 1).numpy()
+    assert np.allclose(rot[0], 1.0)
+    gw = w.shape.grid_w
+    q = 4
+    for (i, j, dr, dc) in [(3, 12, 2, 1), (10, 1, 4, 3), (20, 20, 1, 2)]:
+        i2, j2 = i + dr * gw + dc, j + dr * gw + dc
+        # stay on the same grid row after the column shift
+        if (i - 1) % gw + dc >= gw or (j - 1) % gw + dc >= gw:
+            continue
+        a = rot[i] * np.conj(rot[j])
+        b = rot[i2] * np.conj(rot[j2])
+        assert np.allclose(a, b, atol=1e-12)
+    # and the oracle agrees with the restatement on a full forward (see the first test), whose
+    # attention uses these factors; here: moving a token to another position changes the logits
+    m = O.Model(w.shape, img)
+    s1 = _seq(w.shape, 12, 5)
+    s2 = s1.copy()
+    s2[[3, 9]] = s2[[9, 3]]
+    assert np.abs(m.forward_full(0, s1)[-1] - m.forward_full(0, s2)[-1]).max() > 1e-4
+
+
+def test_synthetic_head_entropy_near_target(tiny, tiny_bf16):
+    for w, img in (tiny, tiny_bf16):
+        m = O.Model(w.shape, img)
+        seq = _seq(w.shape, 40, 6)
+        lg = m.forward_full(1, seq).astype(np.float64)
+        lg -= lg.max(1, keepdims=True)
+        p = np.exp(lg)
+        p /= p.sum(1, keepdims=True)
+        H = -(p * np.log(np.maximum(p, 1e-300))).sum(1).mean()
+        assert abs(H - 3.0) < 0.35, H
