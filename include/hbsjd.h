@@ -1,0 +1,186 @@
+/*
+ * hbsjd.h -- C ABI of the batched speculative-Jacobi rollout library for NVIDIA B200 (sm_100a).
+ *
+ * The library replaces the token-by-token student rollout of visual on-policy
+ * distillation: given a real prefix x_1..x_k per image and its class, it samples
+ * x_{k+1}..x_T from the student (Eq. 2), using independent per-image Jacobi
+ * windows verified in batched forwards (Sec. 4.2) with Full / Compact execution
+ * switching as images finish (Sec. 4.3, Eq. 6).
+ *
+ * General conventions
+ *   - Every function returns 0 (HBSJD_OK) or a negative error code; nothing
+ *     aborts or throws across this boundary.  hbsjd_strerror() names a code and
+ *     hbsjd_last_error(ctx) gives a one-line detail of the last failure.
+ *   - "device" pointers are CUDA global-memory addresses of the context's GPU;
+ *     "host" pointers are ordinary process memory.  The caller owns every
+ *     argument buffer; the context owns weights, KV pages, rollout state and
+ *     all scratch, allocated in hbsjd_create and freed in hbsjd_destroy.
+ *   - All GPU work is enqueued on the stream given to hbsjd_create (a
+ *     cudaStream_t passed as void*, NULL = the legacy default stream).  Calls
+ *     that report a live count synchronise that stream before returning.
+ *   - A context is not thread-safe; use one context per host thread / stream.
+ *   - There is no CPU path: if no CUDA device is usable the calls fail with
+ *     HBSJD_ECUDA.
+ */
+#ifndef HBSJD_H_
+#define HBSJD_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    HBSJD_OK = 0,
+    HBSJD_EINVAL = -1,   /* bad argument; no kernel was launched */
+    HBSJD_ENOMEM = -2,   /* device or host allocation failed */
+    HBSJD_ECUDA = -3,    /* a CUDA call failed (detail in hbsjd_last_error) */
+    HBSJD_ESTATE = -4,   /* call not valid in the context's current state */
+    HBSJD_ETIMEOUT = -5  /* a bounded device-side wait gave up; the context stays usable */
+};
+
+enum { HBSJD_DTYPE_FP32 = 0, HBSJD_DTYPE_BF16 = 1 };
+enum { HBSJD_VERIFY_PROB = 0, HBSJD_VERIFY_GREEDY = 1 };              /* Eq. 5 / Eq. 4 */
+enum { HBSJD_EXEC_FULL = 0, HBSJD_EXEC_COMPACT = 1, HBSJD_EXEC_HYBRID = 2 };  /* Sec. 4.3 */
+
+typedef struct hbsjd_ctx hbsjd_ctx;
+
+/* Decoder description.  Pre-norm blocks: h += Wo Attn(rope(Wq a), rope(Wk a), Wv a), a = rmsnorm(h) g_attn;
+ * h += W2 (silu(W1 m) * (W3 m)), m = rmsnorm(h) g_ffn; logits = W_head rmsnorm(h) g_out.
+ * Sequence index 0 is the class token, index s >= 1 is image token x_s on a grid_h x grid_w raster;
+ * T = grid_h * grid_w tokens per image.  The paper names the model family only (Sec. 5.1). */
+typedef struct {
+    int32_t n_layers, dim, n_heads, ffn_hidden, vocab, grid_h, grid_w, n_classes;
+    int32_t dtype;      /* HBSJD_DTYPE_*: element type of the weight image and of activations */
+    float rms_eps;
+    float rope_base;
+} hbsjd_model_desc;
+
+/* Rollout parameters. */
+typedef struct {
+    int32_t window;          /* W: inputs per image per round = last committed token + W-1 drafts (Sec. 4.2) */
+    int32_t history_offset;  /* H: new draft slots copy the token H positions back (Sec. 4.2) */
+    float cfg_scale;         /* 1 = no guidance; otherwise logits = l_u + s (l_c - l_u) (Sec. 4.2) */
+    float temperature;       /* > 0 */
+    int32_t top_k;           /* 0 or >= vocab: off; ties at the k-th value are kept */
+    int32_t verify_mode;     /* HBSJD_VERIFY_* */
+    int32_t exec_mode;       /* HBSJD_EXEC_* */
+    int32_t gamma;           /* HYBRID: Full iff live images > gamma, else Compact (Eq. 6) */
+    uint64_t seed;           /* key of the counter-based generator; counter = (image, position, round) */
+    int32_t max_rounds;      /* < 0: run to completion; 0: init + prefill only; > 0: at most that many rounds */
+    int32_t reserved;
+} hbsjd_params;
+
+typedef struct {
+    int64_t rounds;            /* verification rounds run with at least one live image */
+    int64_t image_forwards;    /* sum over rounds of live images */
+    int64_t committed;         /* tokens committed (accepted drafts + replacement / bonus tokens) */
+    int64_t rejects;           /* image-rounds that ended in a rejection */
+    int64_t full_rounds;       /* rounds executed in Full form */
+    int64_t compact_rounds;    /* rounds executed in Compact form */
+    int64_t prefill_forwards;  /* batched forwards spent on prefix pre-filling */
+    int64_t kernel_launches;   /* kernels of this library launched by the call */
+    float ms_total;            /* GPU time of the call (CUDA events on the context's stream) */
+    float ms_prefill;          /* of which state init + prefix pre-filling */
+} hbsjd_stats;
+
+/* Creates a context on the current CUDA device.
+ *   m            model description
+ *   weights      HOST pointer to the flat weight image: tok_emb[V,D], cls_emb[C+1,D] (row C = null
+ *                class), per layer g_attn[D], w_qkv[3D,D], w_o[D,D], g_ffn[D], w_13[2F,D], w_2[D,F],
+ *                then g_out[D], w_head[V,D]; matrices row-major [out,in]; each tensor starts on a
+ *                256-byte boundary.  The image is copied; the caller keeps ownership.
+ *   weight_bytes size of the image; must match the description exactly
+ *   max_batch    largest batch of hbsjd_rollout; max_window largest params.window (<= 64)
+ *   cuda_stream  cudaStream_t as void*
+ * Constraints: dim % n_heads == 0, head size 16/32/64/128 (64 for the bf16 tensor-core path),
+ * dim, ffn_hidden, vocab multiples of 64 for bf16.
+ * Errors: HBSJD_EINVAL, HBSJD_ENOMEM, HBSJD_ECUDA. */
+int hbsjd_create(hbsjd_ctx **out, const hbsjd_model_desc *m, const void *weights, size_t weight_bytes,
+                 int max_batch, int max_window, void *cuda_stream);
+
+/* Student rollout of Eq. 2 for `batch` images (Sec. 4.2-4.3).
+ *   prefix_tokens DEVICE int32 [batch, T]; only the first prefix_len[b] entries of row b are read
+ *   prefix_len    DEVICE int32 [batch], 0..T
+ *   class_labels  DEVICE int32 [batch], 0..n_classes-1 (n_classes selects the null class)
+ *   p             HOST parameters
+ *   out_tokens    DEVICE int32 [batch, T]; row b receives x_1..x_T, the prefix copied through.
+ *                 With max_rounds >= 0 positions not yet committed hold drafts / zeros.
+ *   stats         HOST, may be NULL
+ * Runs state init, prefix pre-filling, the initial history windows, then rounds until every image
+ * is complete or max_rounds is reached; returns after the stream has finished that work.
+ * Errors: HBSJD_EINVAL for batch/window beyond the context's limits, prefix_len > T, label or
+ * prefix token out of range, non-positive temperature; HBSJD_ECUDA; HBSJD_ETIMEOUT. */
+int hbsjd_rollout(hbsjd_ctx *c, int batch, const int32_t *prefix_tokens, const int32_t *prefix_len,
+                  const int32_t *class_labels, const hbsjd_params *p, int32_t *out_tokens, hbsjd_stats *stats);
+
+/* hbsjd_rollout for callers whose buffers live in HOST memory (pinned memory makes the copies
+ * asynchronous): copies the three inputs to staging buffers of the context, runs the rollout, and copies
+ * the tokens back, all on the context's stream; returns after the result has arrived.
+ *   prefix_tokens HOST int32 [batch, T];  prefix_len, class_labels HOST int32 [batch];  out_tokens HOST int32 [batch, T] */
+int hbsjd_rollout_host(hbsjd_ctx *c, int batch, const int32_t *prefix_tokens, const int32_t *prefix_len,
+                       const int32_t *class_labels, const hbsjd_params *p, int32_t *out_tokens, hbsjd_stats *stats);
+
+/* One verification round (Sec. 4.2 "Batched verification" .. "Independent progress") on the state left
+ * by hbsjd_rollout or a previous hbsjd_round.  *live_out (HOST) = images still incomplete afterwards.
+ * A sequence of hbsjd_rollout(max_rounds = 0) and hbsjd_round calls yields the same tokens as one
+ * monolithic hbsjd_rollout.  Errors: HBSJD_ESTATE without a preceding hbsjd_rollout. */
+int hbsjd_round(hbsjd_ctx *c, int *live_out);
+
+/* Copies the current token rows (committed tokens, then drafts) to DEVICE int32 [batch, T]. */
+int hbsjd_tokens(hbsjd_ctx *c, int32_t *out_tokens);
+
+/* Frees every resource of the context.  NULL is allowed. */
+void hbsjd_destroy(hbsjd_ctx *c);
+
+/* ---- state export / import (debugging, parity tests, resuming a rollout); HOST buffers ----
+ * cursor int32[batch]: committed tokens per image (Sec. 4.2 "committed cursor")
+ * seq    int32[batch, T+1]: seq[b][t] = token at position t (1-based; entry 0 unused); t <= cursor committed,
+ *        cursor < t < cursor+window: drafts
+ * delta  uint8[batch, T+1]: 1 where the draft is a history / fallback draft (point-mass proposal)
+ * qbase  int32[batch]: cursor at the start of the previous round (row t-qbase-1 of the previous
+ *        round's probabilities is the proposal of draft t)
+ * round  next round index.
+ * hbsjd_set_state leaves the KV pages and the stored probabilities untouched. */
+int hbsjd_get_state(hbsjd_ctx *c, int32_t *cursor, int32_t *seq, uint8_t *delta, int32_t *qbase, int32_t *round);
+int hbsjd_set_state(hbsjd_ctx *c, const int32_t *cursor, const int32_t *seq, const uint8_t *delta,
+                    const int32_t *qbase, int32_t round);
+
+/* Reads intermediate results of the last round into a HOST buffer.
+ *   HBSJD_DBG_PROBS   index = image: fp32 [window, V] probabilities of the last round
+ *   HBSJD_DBG_LOGITS  index = 2*image + branch (0 conditional, 1 unconditional): fp32 [window, V]
+ *   HBSJD_DBG_SLOTS   index ignored: int32 [3, n_slots] = image, cursor, n of each physical slot; returns n_slots
+ * Returns the number of leading rows that are valid (or n_slots), or a negative error. */
+enum { HBSJD_DBG_PROBS = 0, HBSJD_DBG_LOGITS = 1, HBSJD_DBG_SLOTS = 2 };
+int hbsjd_debug_read(hbsjd_ctx *c, int what, int index, void *host_dst, size_t max_bytes);
+
+/* Decoder GEMM as used by the round (Sec. 4.2 verifier forward): C[M,N] (+)= A[M,K] . W[N,K]^T on the
+ * context's stream.  A, W: DEVICE, element type of the context (bf16: tcgen05 tensor cores, fp32
+ * accumulation; fp32: CUDA cores).  C: DEVICE fp32 [M,N]; accumulate != 0 adds into C.
+ * M may be any size; bf16 needs N % 64 == 0 and K % 64 == 0; A, W 16-byte aligned. */
+int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate);
+
+/* Per-kernel-class timing with CUDA events on the context's stream (off by default).  While enabled,
+ * every launch of a timed class is bracketed by an event pair; totals accumulate until the next
+ * hbsjd_profile(c, 1), which also resets them.  work = algorithmic FLOPs (GEMM: 2 M N K per launch) or
+ * algorithmic bytes (attention: K,V rows read + q read + output written; accept: logits read + probabilities
+ * written) of the launches that were timed. */
+enum { HBSJD_PROF_GEMM = 0, HBSJD_PROF_ATTENTION = 1, HBSJD_PROF_ACCEPT = 2, HBSJD_PROF_OTHER = 3 };
+typedef struct {
+    double ms[4];
+    double work[4];
+    int64_t launches[4];
+    int64_t dropped;   /* launches not timed because the event pool was exhausted */
+} hbsjd_kernel_profile;
+int hbsjd_profile(hbsjd_ctx *c, int enable);
+int hbsjd_profile_read(hbsjd_ctx *c, hbsjd_kernel_profile *out);
+
+const char *hbsjd_strerror(int code);
+const char *hbsjd_last_error(const hbsjd_ctx *c);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HBSJD_H_ */

@@ -1,0 +1,752 @@
+// C ABI of the rollout library (see include/hbsjd.h): context, host-side round loop, debug helpers.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <type_traits>
+#include <vector>
+
+#include "../../include/hbsjd.h"
+#include "internal.h"
+
+using namespace hbsjd;
+
+namespace {
+
+constexpr int PAGE_TOKENS = 64;
+
+struct LayerW {
+    const void *g_attn, *w_qkv, *w_o, *g_ffn, *w_13, *w_2;
+};
+
+}  // namespace
+
+struct hbsjd_ctx {
+    hbsjd_model_desc d;
+    int T, dh, Bmax, Wmax;
+    bool bf16_model;
+    bool simt_gemm;      // debugging: run the bf16 GEMMs on CUDA cores
+    bool ref_attention;  // debugging: run the one-warp-per-row attention kernel
+    cudaStream_t stream;
+    // weights
+    unsigned char* w_img;
+    const void *tok_emb, *cls_emb, *g_out, *w_head;
+    std::vector<LayerW> layers;
+    float* rope_cs;
+    // KV pages
+    void *kc, *vc;
+    int32_t* page_table;
+    int pages_per_row, n_pages;
+    // rollout state
+    State st;
+    float* pbuf[2];
+    int parity;
+    uint8_t* flag;
+    int32_t *cand_rep, *cand_ref;
+    // activations
+    float *h, *qkv, *gu, *logits;
+    void *a, *q, *o, *act;
+    // host side
+    int32_t* h_counters;  // pinned [8]
+    cudaEvent_t ev0, ev1, ev2;
+    hbsjd_params P;
+    bool have_rollout;
+    int live, round, last_S, last_compact;
+    hbsjd_stats stats;
+    long long launches;
+    // host-buffer staging
+    int32_t *stage_tok, *stage_len, *stage_lab, *stage_out;
+    // per-class event timing
+    bool profiling;
+    struct ProfSlot { cudaEvent_t a, b; int cls; double work; };
+    std::vector<ProfSlot> pool;
+    int pool_used;
+    int pending_attn;  // attention launches of the current forward whose byte count waits for the counters
+    hbsjd_kernel_profile prof;
+    char err[256];
+};
+
+namespace {
+
+#define CK(call)                                                                                  \
+    do {                                                                                          \
+        cudaError_t e_ = (call);                                                                  \
+        if (e_ != cudaSuccess) {                                                                  \
+            snprintf(c->err, sizeof(c->err), "%s: %s", #call, cudaGetErrorString(e_));            \
+            return e_ == cudaErrorMemoryAllocation ? HBSJD_ENOMEM : HBSJD_ECUDA;                  \
+        }                                                                                         \
+    } while (0)
+
+size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// Brackets the launches issued between prof_begin and prof_end with an event pair of class `cls`.
+int prof_begin(hbsjd_ctx* c, int cls, double work) {
+    if (!c->profiling) return -1;
+    if (c->pool_used >= (int)c->pool.size()) {
+        c->prof.dropped++;
+        return -1;
+    }
+    hbsjd_ctx::ProfSlot& s = c->pool[c->pool_used];
+    s.cls = cls;
+    s.work = work;
+    cudaEventRecord(s.a, c->stream);
+    return c->pool_used++;
+}
+void prof_end(hbsjd_ctx* c, int slot) {
+    if (slot >= 0) cudaEventRecord(c->pool[slot].b, c->stream);
+}
+// After a stream synchronisation: folds the finished event pairs into the totals.  attn_bytes is the
+// algorithmic traffic of each attention launch of the forward just finished.
+void prof_resolve(hbsjd_ctx* c, double attn_bytes, double accept_bytes) {
+    for (int i = 0; i < c->pool_used; ++i) {
+        hbsjd_ctx::ProfSlot& s = c->pool[i];
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, s.a, s.b) != cudaSuccess) continue;
+        double work = s.work;
+        if (s.cls == HBSJD_PROF_ATTENTION) work = attn_bytes;
+        if (s.cls == HBSJD_PROF_ACCEPT) work = accept_bytes;
+        c->prof.ms[s.cls] += ms;
+        c->prof.work[s.cls] += work;
+        c->prof.launches[s.cls] += 1;
+    }
+    c->pool_used = 0;
+}
+
+template <typename T>
+int dev_alloc(hbsjd_ctx* c, T** p, size_t count) {
+    *p = nullptr;
+    CK(cudaMalloc((void**)p, count * sizeof(T) > 0 ? count * sizeof(T) : 16));
+    CK(cudaMemsetAsync(*p, 0, count * sizeof(T), c->stream));
+    return 0;
+}
+
+KvView kv_view(const hbsjd_ctx* c) {
+    KvView kv;
+    kv.k = c->kc;
+    kv.v = c->vc;
+    kv.table = c->page_table;
+    kv.pages_per_row = c->pages_per_row;
+    kv.page = PAGE_TOKENS;
+    kv.n_pages = c->n_pages;
+    kv.D = c->d.dim;
+    return kv;
+}
+
+template <typename TA>
+int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate);
+
+template <>
+int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
+    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
+    launch_gemm_simt<float>((const float*)A, (const float*)W, C, M, N, K, accumulate, c->stream);
+    prof_end(c, ps);
+    c->launches++;
+    return 0;
+}
+
+template <>
+int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
+    c->launches++;
+    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
+    if (c->simt_gemm) {
+        launch_gemm_simt<bf16>((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, c->stream);
+        prof_end(c, ps);
+        return 0;
+    }
+    const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, 0,
+                                    c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err));
+    prof_end(c, ps);
+    return rc == 0 ? 0 : (rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA);
+}
+
+// One batched verifier forward over S slots (Sec. 4.2 "Batched verification").
+template <typename TA>
+int forward(hbsjd_ctx* c, int S, bool want_logits) {
+    const State& st = c->st;
+    const int M = st.nb * S * st.W, D = st.D, F = st.F;
+    cudaStream_t s = c->stream;
+    const KvView kv = kv_view(c);
+    launch_embed<TA>(st, S, (const TA*)c->tok_emb, (const TA*)c->cls_emb, c->h, s);
+    c->launches++;
+    for (int l = 0; l < st.L; ++l) {
+        const LayerW& w = c->layers[l];
+        int rc;
+        launch_rmsnorm<TA>(c->h, (const TA*)w.g_attn, (TA*)c->a, M, D, c->d.rms_eps, s);
+        if ((rc = gemm<TA>(c, c->a, w.w_qkv, c->qkv, M, 3 * D, D, 0))) return rc;
+        launch_rope_kv<TA>(st, S, l, c->qkv, c->rope_cs, (TA*)c->q, kv, s);
+        {
+            const int ps = prof_begin(c, HBSJD_PROF_ATTENTION, 0.0);
+            if constexpr (std::is_same<TA, bf16>::value) {
+                if (!c->ref_attention && attention_mma_supported(st, kv))
+                    launch_attention_mma(st, S, l, (const bf16*)c->q, kv, (bf16*)c->o, s);
+                else
+                    launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
+            } else {
+                launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
+            }
+            prof_end(c, ps);
+        }
+        if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1))) return rc;
+        launch_rmsnorm<TA>(c->h, (const TA*)w.g_ffn, (TA*)c->a, M, D, c->d.rms_eps, s);
+        if ((rc = gemm<TA>(c, c->a, w.w_13, c->gu, M, 2 * F, D, 0))) return rc;
+        launch_swiglu<TA>(c->gu, (TA*)c->act, M, F, s);
+        if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1))) return rc;
+        c->launches += 5;
+    }
+    if (want_logits) {
+        launch_rmsnorm<TA>(c->h, (const TA*)c->g_out, (TA*)c->a, M, D, c->d.rms_eps, s);
+        c->launches++;
+        int rc;
+        if ((rc = gemm<TA>(c, c->a, c->w_head, c->logits, M, st.V, D, 0))) return rc;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        snprintf(c->err, sizeof(c->err), "forward launch: %s", cudaGetErrorString(e));
+        return HBSJD_ECUDA;
+    }
+    return 0;
+}
+
+int forward_any(hbsjd_ctx* c, int S, bool want_logits) {
+    return c->bf16_model ? forward<bf16>(c, S, want_logits) : forward<float>(c, S, want_logits);
+}
+
+int choose_compact(const hbsjd_ctx* c, int live) {
+    if (c->P.exec_mode == HBSJD_EXEC_FULL) return 0;
+    if (c->P.exec_mode == HBSJD_EXEC_COMPACT) return 1;
+    return live > c->P.gamma ? 0 : 1;  // Eq. 6
+}
+
+int sync_counters(hbsjd_ctx* c) {
+    CK(cudaMemcpyAsync(c->h_counters, c->st.counters, 8 * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (c->profiling) {
+        // algorithmic bytes of the forward just finished, from the slot set-up sums:
+        // attention per layer: K and V rows 0..c+n-1 read per row, q read and output written per input;
+        // accept: logits of every branch read, probabilities written, per input
+        const double es = c->bf16_model ? 2.0 : 4.0, D = c->d.dim, V = c->d.vocab, nb = c->st.nb;
+        const double keys = c->h_counters[CNT_SUM_KEYS], n = c->h_counters[CNT_SUM_N];
+        prof_resolve(c, nb * (keys * 2.0 * D * es + n * 2.0 * D * es), n * (nb + 1.0) * V * 4.0);
+    }
+    if (c->h_counters[CNT_ERROR] != 0) {
+        snprintf(c->err, sizeof(c->err), "a bounded device-side wait gave up (code %d)", c->h_counters[CNT_ERROR]);
+        cudaMemsetAsync(c->st.counters + CNT_ERROR, 0, sizeof(int32_t), c->stream);
+        return HBSJD_ETIMEOUT;
+    }
+    return 0;
+}
+
+int run_round(hbsjd_ctx* c) {
+    if (c->live == 0) return 0;
+    const int compact = choose_compact(c, c->live);
+    const int S = compact ? c->live : c->st.B;
+    launch_setup(c->st, 0, compact, c->stream);
+    c->launches++;
+    int rc = forward_any(c, S, true);
+    if (rc) return rc;
+    AcceptArgs a;
+    a.logits = c->logits;
+    a.pcur = c->pbuf[c->parity];
+    a.pprev = c->pbuf[c->parity ^ 1];
+    a.flag = c->flag;
+    a.cand_rep = c->cand_rep;
+    a.cand_ref = c->cand_ref;
+    a.S = S;
+    a.cfg_scale = c->P.cfg_scale;
+    a.temperature = c->P.temperature;
+    a.top_k = c->P.top_k;
+    a.greedy = c->P.verify_mode == HBSJD_VERIFY_GREEDY;
+    a.seed_lo = (uint32_t)(c->P.seed & 0xffffffffu);
+    a.seed_hi = (uint32_t)(c->P.seed >> 32);
+    a.round = (uint32_t)c->round;
+    {
+        const int ps = prof_begin(c, HBSJD_PROF_ACCEPT, 0.0);
+        launch_prob_accept(c->st, a, c->stream);
+        launch_commit(c->st, a, c->stream);
+        prof_end(c, ps);
+    }
+    c->launches += 2;
+    CK(cudaGetLastError());
+    rc = sync_counters(c);
+    if (rc) return rc;
+    if (c->h_counters[CNT_LIVE_SETUP] != c->live) {
+        snprintf(c->err, sizeof(c->err), "live count mismatch: host %d device %d", c->live,
+                 c->h_counters[CNT_LIVE_SETUP]);
+        return HBSJD_ESTATE;
+    }
+    c->stats.rounds += 1;
+    c->stats.image_forwards += c->live;
+    if (compact) c->stats.compact_rounds += 1;
+    else c->stats.full_rounds += 1;
+    c->stats.committed = c->h_counters[CNT_COMMITTED];
+    c->stats.rejects = c->h_counters[CNT_REJECTS];
+    c->live = c->h_counters[CNT_LIVE];
+    c->last_S = S;
+    c->last_compact = compact;
+    c->round += 1;
+    c->parity ^= 1;
+    return 0;
+}
+
+void free_all(hbsjd_ctx* c) {
+    void* ptrs[] = {c->w_img, c->rope_cs, c->kc, c->vc, c->page_table, c->st.cursor, c->st.seq, c->st.delta,
+                    c->st.qbase, c->st.label, c->st.klen, c->st.pfill, c->st.slot_img, c->st.slot_c, c->st.slot_n,
+                    c->st.counters, c->st.m_last, c->st.j_last, c->pbuf[0], c->pbuf[1], c->flag, c->cand_rep,
+                    c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act,
+                    c->stage_tok, c->stage_len, c->stage_lab, c->stage_out};
+    for (void* p : ptrs)
+        if (p) cudaFree(p);
+    if (c->h_counters) cudaFreeHost(c->h_counters);
+    for (auto& s : c->pool) {
+        if (s.a) cudaEventDestroy(s.a);
+        if (s.b) cudaEventDestroy(s.b);
+    }
+    if (c->ev0) cudaEventDestroy(c->ev0);
+    if (c->ev1) cudaEventDestroy(c->ev1);
+    if (c->ev2) cudaEventDestroy(c->ev2);
+}
+
+int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
+    const hbsjd_model_desc& d = c->d;
+    const size_t D = d.dim, F = d.ffn_hidden, V = d.vocab, L = d.n_layers;
+    const size_t es = c->bf16_model ? 2 : 4;
+    // weight image offsets (each tensor on a 256-byte boundary)
+    size_t off = 0;
+    auto take = [&](size_t count) {
+        const size_t o = off;
+        off = align256(off + count * es);
+        return o;
+    };
+    const size_t o_tok = take(V * D), o_cls = take((size_t)(d.n_classes + 1) * D);
+    std::vector<size_t> lo(L * 6);
+    for (size_t l = 0; l < L; ++l) {
+        lo[l * 6 + 0] = take(D);
+        lo[l * 6 + 1] = take(3 * D * D);
+        lo[l * 6 + 2] = take(D * D);
+        lo[l * 6 + 3] = take(D);
+        lo[l * 6 + 4] = take(2 * F * D);
+        lo[l * 6 + 5] = take(D * F);
+    }
+    const size_t o_gout = take(D), o_head = take(V * D);
+    if (off != weight_bytes) {
+        snprintf(c->err, sizeof(c->err), "weight image is %zu bytes, the description needs %zu", weight_bytes, off);
+        return HBSJD_EINVAL;
+    }
+    CK(cudaMalloc((void**)&c->w_img, off));
+    CK(cudaMemcpyAsync(c->w_img, weights, off, cudaMemcpyHostToDevice, c->stream));
+    c->tok_emb = c->w_img + o_tok;
+    c->cls_emb = c->w_img + o_cls;
+    c->g_out = c->w_img + o_gout;
+    c->w_head = c->w_img + o_head;
+    c->layers.resize(L);
+    for (size_t l = 0; l < L; ++l) {
+        c->layers[l].g_attn = c->w_img + lo[l * 6 + 0];
+        c->layers[l].w_qkv = c->w_img + lo[l * 6 + 1];
+        c->layers[l].w_o = c->w_img + lo[l * 6 + 2];
+        c->layers[l].g_ffn = c->w_img + lo[l * 6 + 3];
+        c->layers[l].w_13 = c->w_img + lo[l * 6 + 4];
+        c->layers[l].w_2 = c->w_img + lo[l * 6 + 5];
+    }
+    // 2D rotary table by sequence index: index 0 unrotated; index s >= 1 at (row, col) of the raster
+    {
+        const int half = c->dh / 2, quarter = c->dh / 4;
+        std::vector<float> tab((size_t)c->T * half * 2);
+        for (int s = 0; s < c->T; ++s)
+            for (int e = 0; e < half; ++e) {
+                double ang = 0.0;
+                if (s > 0) {
+                    const int row = (s - 1) / d.grid_w, col = (s - 1) % d.grid_w;
+                    const int ee = e < quarter ? e : e - quarter;
+                    const double w = std::pow((double)d.rope_base, -(double)ee / (double)quarter);
+                    ang = (e < quarter ? (double)row : (double)col) * w;
+                }
+                tab[((size_t)s * half + e) * 2] = (float)std::cos(ang);
+                tab[((size_t)s * half + e) * 2 + 1] = (float)std::sin(ang);
+            }
+        CK(cudaMalloc((void**)&c->rope_cs, tab.size() * sizeof(float)));
+        CK(cudaMemcpyAsync(c->rope_cs, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+    }
+    // KV pages: two cache rows (conditional, unconditional) per image
+    const int rows = 2 * c->Bmax;
+    c->pages_per_row = (c->T + PAGE_TOKENS - 1) / PAGE_TOKENS;
+    c->n_pages = rows * c->pages_per_row;
+    const size_t kv_elems = L * (size_t)c->n_pages * PAGE_TOKENS * D;
+    CK(cudaMalloc(&c->kc, kv_elems * es));
+    CK(cudaMalloc(&c->vc, kv_elems * es));
+    CK(cudaMemsetAsync(c->kc, 0, kv_elems * es, c->stream));
+    CK(cudaMemsetAsync(c->vc, 0, kv_elems * es, c->stream));
+    {
+        std::vector<int32_t> tab(c->n_pages);
+        for (int i = 0; i < c->n_pages; ++i) tab[i] = i;
+        const char* sh = getenv("HBSJD_PAGE_SHUFFLE");
+        if (sh && atoi(sh) != 0) {  // scatter the pages (exercises the page-table indirection)
+            uint64_t x = 0x9E3779B97F4A7C15ull * (uint64_t)atoi(sh);
+            for (int i = c->n_pages - 1; i > 0; --i) {
+                x = x * 6364136223846793005ull + 1442695040888963407ull;
+                const int j = (int)((x >> 33) % (uint64_t)(i + 1));
+                std::swap(tab[i], tab[j]);
+            }
+        }
+        CK(cudaMalloc((void**)&c->page_table, tab.size() * sizeof(int32_t)));
+        CK(cudaMemcpyAsync(c->page_table, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
+                           c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+    }
+    // state
+    const size_t Bm = c->Bmax, Wm = c->Wmax, T1 = c->T + 1;
+    int rc;
+    State& st = c->st;
+    if ((rc = dev_alloc(c, &st.cursor, Bm)) || (rc = dev_alloc(c, &st.seq, Bm * T1)) ||
+        (rc = dev_alloc(c, &st.delta, Bm * T1)) || (rc = dev_alloc(c, &st.qbase, Bm)) ||
+        (rc = dev_alloc(c, &st.label, Bm)) || (rc = dev_alloc(c, &st.klen, Bm)) ||
+        (rc = dev_alloc(c, &st.pfill, Bm)) || (rc = dev_alloc(c, &st.slot_img, Bm)) ||
+        (rc = dev_alloc(c, &st.slot_c, Bm)) || (rc = dev_alloc(c, &st.slot_n, Bm)) ||
+        (rc = dev_alloc(c, &st.counters, (size_t)8)) || (rc = dev_alloc(c, &st.m_last, Bm)) ||
+        (rc = dev_alloc(c, &st.j_last, Bm)) || (rc = dev_alloc(c, &c->pbuf[0], Bm * Wm * V)) ||
+        (rc = dev_alloc(c, &c->pbuf[1], Bm * Wm * V)) || (rc = dev_alloc(c, &c->flag, Bm * Wm)) ||
+        (rc = dev_alloc(c, &c->cand_rep, Bm * Wm)) || (rc = dev_alloc(c, &c->cand_ref, Bm * Wm)))
+        return rc;
+    // activations for the largest forward: 2 branches x max_batch slots x max_window inputs
+    const size_t Mmax = 2 * Bm * Wm;
+    unsigned char *a, *q, *o, *act;
+    if ((rc = dev_alloc(c, &c->h, Mmax * D)) || (rc = dev_alloc(c, &c->qkv, Mmax * 3 * D)) ||
+        (rc = dev_alloc(c, &c->gu, Mmax * 2 * F)) || (rc = dev_alloc(c, &c->logits, Mmax * V)) ||
+        (rc = dev_alloc(c, &a, Mmax * D * es)) || (rc = dev_alloc(c, &q, Mmax * D * es)) ||
+        (rc = dev_alloc(c, &o, Mmax * D * es)) || (rc = dev_alloc(c, &act, Mmax * F * es)))
+        return rc;
+    c->a = a;
+    c->q = q;
+    c->o = o;
+    c->act = act;
+    if ((rc = dev_alloc(c, &c->stage_tok, Bm * (size_t)c->T)) || (rc = dev_alloc(c, &c->stage_len, Bm)) ||
+        (rc = dev_alloc(c, &c->stage_lab, Bm)) || (rc = dev_alloc(c, &c->stage_out, Bm * (size_t)c->T)))
+        return rc;
+    c->pool.resize(1024);
+    for (auto& s : c->pool) {
+        s.a = s.b = nullptr;
+        CK(cudaEventCreate(&s.a));
+        CK(cudaEventCreate(&s.b));
+    }
+    CK(cudaMallocHost((void**)&c->h_counters, 8 * sizeof(int32_t)));
+    CK(cudaEventCreate(&c->ev0));
+    CK(cudaEventCreate(&c->ev1));
+    CK(cudaEventCreate(&c->ev2));
+    CK(cudaStreamSynchronize(c->stream));
+    return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* hbsjd_strerror(int code) {
+    switch (code) {
+        case HBSJD_OK: return "ok";
+        case HBSJD_EINVAL: return "invalid argument";
+        case HBSJD_ENOMEM: return "out of memory";
+        case HBSJD_ECUDA: return "CUDA error";
+        case HBSJD_ESTATE: return "call not valid in this state";
+        case HBSJD_ETIMEOUT: return "bounded device wait gave up";
+        default: return "unknown error";
+    }
+}
+
+const char* hbsjd_last_error(const hbsjd_ctx* c) { return c ? c->err : "null context"; }
+
+int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights, size_t weight_bytes,
+                 int max_batch, int max_window, void* cuda_stream) {
+    if (!out) return HBSJD_EINVAL;
+    *out = nullptr;
+    if (!m || !weights) return HBSJD_EINVAL;
+    if (m->n_layers < 1 || m->dim < 16 || m->n_heads < 1 || m->dim % m->n_heads != 0 || m->ffn_hidden < 16 ||
+        m->vocab < 4 || m->vocab % 4 != 0 || m->grid_h < 1 || m->grid_w < 1 || m->n_classes < 1 ||
+        (m->dtype != HBSJD_DTYPE_FP32 && m->dtype != HBSJD_DTYPE_BF16) || !(m->rms_eps > 0) || !(m->rope_base > 1) ||
+        max_batch < 1 || max_window < 1 || max_window > 64)
+        return HBSJD_EINVAL;
+    const int dh = m->dim / m->n_heads;
+    if (dh != 16 && dh != 32 && dh != 64 && dh != 128) return HBSJD_EINVAL;
+    if (m->dim % 16 || m->ffn_hidden % 16) return HBSJD_EINVAL;
+    if (m->dtype == HBSJD_DTYPE_BF16 && (m->dim % 64 || m->ffn_hidden % 64 || m->vocab % 64)) return HBSJD_EINVAL;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return HBSJD_ECUDA;
+    hbsjd_ctx* c = new (std::nothrow) hbsjd_ctx();
+    if (!c) return HBSJD_ENOMEM;
+    memset((void*)&c->st, 0, sizeof(State));
+    c->d = *m;
+    c->T = m->grid_h * m->grid_w;
+    c->dh = dh;
+    c->Bmax = max_batch;
+    c->Wmax = max_window;
+    c->bf16_model = m->dtype == HBSJD_DTYPE_BF16;
+    const char* g = getenv("HBSJD_GEMM");
+    c->simt_gemm = g && strcmp(g, "simt") == 0;
+    const char* at = getenv("HBSJD_ATTENTION");
+    c->ref_attention = at && strcmp(at, "ref") == 0;
+    c->stream = (cudaStream_t)cuda_stream;
+    c->err[0] = 0;
+    const int rc = create_impl(c, weights, weight_bytes);
+    if (rc != 0) {
+        fprintf(stderr, "hbsjd_create: %s\n", c->err);
+        free_all(c);
+        delete c;
+        return rc;
+    }
+    *out = c;
+    return HBSJD_OK;
+}
+
+void hbsjd_destroy(hbsjd_ctx* c) {
+    if (!c) return;
+    cudaStreamSynchronize(c->stream);
+    free_all(c);
+    delete c;
+}
+
+int hbsjd_rollout(hbsjd_ctx* c, int batch, const int32_t* prefix_tokens, const int32_t* prefix_len,
+                  const int32_t* class_labels, const hbsjd_params* p, int32_t* out_tokens, hbsjd_stats* stats) {
+    if (!c) return HBSJD_EINVAL;
+    c->err[0] = 0;
+    if (!prefix_tokens || !prefix_len || !class_labels || !p || !out_tokens) {
+        snprintf(c->err, sizeof(c->err), "null argument");
+        return HBSJD_EINVAL;
+    }
+    if (batch < 1 || batch > c->Bmax || p->window < 1 || p->window > c->Wmax || p->history_offset < 1 ||
+        !(p->temperature > 0.f) || !std::isfinite(p->cfg_scale) || p->top_k < 0 ||
+        (p->verify_mode != HBSJD_VERIFY_PROB && p->verify_mode != HBSJD_VERIFY_GREEDY) ||
+        p->exec_mode < HBSJD_EXEC_FULL || p->exec_mode > HBSJD_EXEC_HYBRID || p->gamma < 0) {
+        snprintf(c->err, sizeof(c->err), "parameter out of range (batch %d window %d)", batch, p->window);
+        return HBSJD_EINVAL;
+    }
+    const int T = c->T, V = c->d.vocab;
+    // validate the integer inputs on the host before any kernel runs
+    std::vector<int32_t> hk(batch), hl(batch), ht((size_t)batch * T);
+    CK(cudaMemcpyAsync(hk.data(), prefix_len, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(hl.data(), class_labels, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(ht.data(), prefix_tokens, (size_t)batch * T * sizeof(int32_t), cudaMemcpyDeviceToHost,
+                       c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    int kmax = 0, live = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (hk[b] < 0 || hk[b] > T || hl[b] < 0 || hl[b] > c->d.n_classes) {
+            snprintf(c->err, sizeof(c->err), "image %d: prefix_len %d or label %d out of range", b, hk[b], hl[b]);
+            return HBSJD_EINVAL;
+        }
+        for (int t = 0; t < hk[b]; ++t)
+            if (ht[(size_t)b * T + t] < 0 || ht[(size_t)b * T + t] >= V) {
+                snprintf(c->err, sizeof(c->err), "image %d: prefix token %d out of range", b, t);
+                return HBSJD_EINVAL;
+            }
+        kmax = hk[b] > kmax ? hk[b] : kmax;
+        live += hk[b] < T;
+    }
+    c->P = *p;
+    State& st = c->st;
+    st.B = batch;
+    st.T = T;
+    st.V = V;
+    st.D = c->d.dim;
+    st.Hh = c->d.n_heads;
+    st.dh = c->dh;
+    st.F = c->d.ffn_hidden;
+    st.L = c->d.n_layers;
+    st.C = c->d.n_classes;
+    st.Bmax = c->Bmax;
+    st.Wmax = c->Wmax;
+    st.W = p->window;
+    st.H = p->history_offset;
+    st.nb = p->cfg_scale != 1.0f ? 2 : 1;
+    memset(&c->stats, 0, sizeof(c->stats));
+    c->launches = 0;
+    c->round = 0;
+    c->parity = 0;
+    c->live = live;
+    c->have_rollout = false;
+
+    CK(cudaEventRecord(c->ev0, c->stream));
+    launch_init_state(st, prefix_tokens, prefix_len, class_labels, c->stream);
+    c->launches++;
+    // prefix pre-filling: cache sequence indices 0..k-1 in chunks of W (no LM head)
+    for (int pr = 0;; ++pr) {
+        int act = 0;
+        for (int b = 0; b < batch; ++b) act += hk[b] > pr * p->window;
+        if (act == 0) break;
+        const int compact = choose_compact(c, act);
+        const int S = compact ? act : batch;
+        launch_setup(st, 1, compact, c->stream);
+        const int rc = forward_any(c, S, false);
+        if (rc) return rc;
+        launch_prefill_advance(st, S, c->stream);
+        c->launches += 2;
+        c->stats.prefill_forwards += 1;
+        if (c->profiling) {  // fold this forward's event pairs while its byte counters are current
+            const int rs = sync_counters(c);
+            if (rs) return rs;
+        }
+    }
+    launch_init_window(st, (uint32_t)(p->seed & 0xffffffffu), (uint32_t)(p->seed >> 32), c->stream);
+    c->launches++;
+    CK(cudaEventRecord(c->ev1, c->stream));
+    if (c->profiling) {
+        const int rc = sync_counters(c);
+        if (rc) return rc;
+    }
+    CK(cudaGetLastError());
+    c->have_rollout = true;
+
+    int rounds = 0;
+    while (c->live > 0 && (p->max_rounds < 0 || rounds < p->max_rounds)) {
+        const int rc = run_round(c);
+        if (rc) return rc;
+        ++rounds;
+    }
+    launch_export_tokens(st, out_tokens, c->stream);
+    c->launches++;
+    CK(cudaEventRecord(c->ev2, c->stream));
+    const int rc = sync_counters(c);
+    if (rc) return rc;
+    CK(cudaEventElapsedTime(&c->stats.ms_prefill, c->ev0, c->ev1));
+    CK(cudaEventElapsedTime(&c->stats.ms_total, c->ev0, c->ev2));
+    c->stats.kernel_launches = c->launches;
+    if (stats) *stats = c->stats;
+    return HBSJD_OK;
+}
+
+int hbsjd_rollout_host(hbsjd_ctx* c, int batch, const int32_t* prefix_tokens, const int32_t* prefix_len,
+                       const int32_t* class_labels, const hbsjd_params* p, int32_t* out_tokens, hbsjd_stats* stats) {
+    if (!c) return HBSJD_EINVAL;
+    if (!prefix_tokens || !prefix_len || !class_labels || !p || !out_tokens || batch < 1 || batch > c->Bmax) {
+        snprintf(c->err, sizeof(c->err), "null argument or batch out of range");
+        return HBSJD_EINVAL;
+    }
+    const size_t bt = (size_t)batch * c->T * sizeof(int32_t), bb = (size_t)batch * sizeof(int32_t);
+    CK(cudaMemcpyAsync(c->stage_tok, prefix_tokens, bt, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->stage_len, prefix_len, bb, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->stage_lab, class_labels, bb, cudaMemcpyHostToDevice, c->stream));
+    const int rc = hbsjd_rollout(c, batch, c->stage_tok, c->stage_len, c->stage_lab, p, c->stage_out, stats);
+    if (rc) return rc;
+    CK(cudaMemcpyAsync(out_tokens, c->stage_out, bt, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
+}
+
+int hbsjd_profile(hbsjd_ctx* c, int enable) {
+    if (!c) return HBSJD_EINVAL;
+    CK(cudaStreamSynchronize(c->stream));
+    c->profiling = enable != 0;
+    c->pool_used = 0;
+    memset(&c->prof, 0, sizeof(c->prof));
+    return HBSJD_OK;
+}
+
+int hbsjd_profile_read(hbsjd_ctx* c, hbsjd_kernel_profile* out) {
+    if (!c || !out) return HBSJD_EINVAL;
+    *out = c->prof;
+    return HBSJD_OK;
+}
+
+int hbsjd_round(hbsjd_ctx* c, int* live_out) {
+    if (!c) return HBSJD_EINVAL;
+    if (!c->have_rollout) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_round needs a preceding hbsjd_rollout");
+        return HBSJD_ESTATE;
+    }
+    const int rc = run_round(c);
+    if (rc) return rc;
+    if (live_out) *live_out = c->live;
+    return HBSJD_OK;
+}
+
+int hbsjd_tokens(hbsjd_ctx* c, int32_t* out_tokens) {
+    if (!c || !out_tokens) return HBSJD_EINVAL;
+    if (!c->have_rollout) return HBSJD_ESTATE;
+    launch_export_tokens(c->st, out_tokens, c->stream);
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
+}
+
+int hbsjd_get_state(hbsjd_ctx* c, int32_t* cursor, int32_t* seq, uint8_t* delta, int32_t* qbase, int32_t* round) {
+    if (!c) return HBSJD_EINVAL;
+    if (!c->have_rollout) return HBSJD_ESTATE;
+    const size_t B = c->st.B, T1 = c->T + 1;
+    if (cursor) CK(cudaMemcpyAsync(cursor, c->st.cursor, B * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (seq) CK(cudaMemcpyAsync(seq, c->st.seq, B * T1 * 4, cudaMemcpyDeviceToHost, c->stream));
+    if (delta) CK(cudaMemcpyAsync(delta, c->st.delta, B * T1, cudaMemcpyDeviceToHost, c->stream));
+    if (qbase) CK(cudaMemcpyAsync(qbase, c->st.qbase, B * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (round) *round = c->round;
+    return HBSJD_OK;
+}
+
+int hbsjd_set_state(hbsjd_ctx* c, const int32_t* cursor, const int32_t* seq, const uint8_t* delta,
+                    const int32_t* qbase, int32_t round) {
+    if (!c || !cursor || !seq || !delta || !qbase) return HBSJD_EINVAL;
+    if (!c->have_rollout) return HBSJD_ESTATE;
+    const size_t B = c->st.B, T1 = c->T + 1;
+    int live = 0;
+    for (size_t b = 0; b < B; ++b) {
+        if (cursor[b] < 0 || cursor[b] > c->T || qbase[b] < 0 || qbase[b] > cursor[b]) {
+            snprintf(c->err, sizeof(c->err), "set_state: image %zu cursor/qbase out of range", b);
+            return HBSJD_EINVAL;
+        }
+        for (size_t t = 1; t < T1; ++t)
+            if (seq[b * T1 + t] < 0 || seq[b * T1 + t] >= c->d.vocab) {
+                snprintf(c->err, sizeof(c->err), "set_state: image %zu token %zu out of range", b, t);
+                return HBSJD_EINVAL;
+            }
+        live += cursor[b] < c->T;
+    }
+    CK(cudaMemcpyAsync(c->st.cursor, cursor, B * 4, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->st.seq, seq, B * T1 * 4, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->st.delta, delta, B * T1, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaMemcpyAsync(c->st.qbase, qbase, B * 4, cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    c->live = live;
+    c->round = round;
+    return HBSJD_OK;
+}
+
+int hbsjd_debug_read(hbsjd_ctx* c, int what, int index, void* host_dst, size_t max_bytes) {
+    if (!c || !host_dst) return HBSJD_EINVAL;
+    if (!c->have_rollout || c->round == 0) return HBSJD_ESTATE;
+    const int S = c->last_S, W = c->st.W, V = c->d.vocab;
+    std::vector<int32_t> slots((size_t)3 * S);
+    CK(cudaMemcpyAsync(slots.data(), c->st.slot_img, S * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(slots.data() + S, c->st.slot_c, S * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(slots.data() + 2 * S, c->st.slot_n, S * 4, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    if (what == HBSJD_DBG_SLOTS) {
+        if (max_bytes < slots.size() * 4) return HBSJD_EINVAL;
+        memcpy(host_dst, slots.data(), slots.size() * 4);
+        return S;
+    }
+    const int img = what == HBSJD_DBG_LOGITS ? index / 2 : index;
+    const int branch = what == HBSJD_DBG_LOGITS ? index % 2 : 0;
+    if (img < 0 || img >= c->st.B || (branch == 1 && c->st.nb == 1)) return HBSJD_EINVAL;
+    int slot = -1;
+    for (int s = 0; s < S; ++s)
+        if (slots[s] == img) slot = s;
+    if (slot < 0) return 0;
+    const int n = slots[2 * S + slot];
+    if (n == 0) return 0;
+    const size_t bytes = (size_t)n * V * sizeof(float);
+    if (max_bytes < bytes) return HBSJD_EINVAL;
+    const float* src;
+    if (what == HBSJD_DBG_PROBS) src = c->pbuf[c->parity ^ 1] + (size_t)img * c->Wmax * V;
+    else if (what == HBSJD_DBG_LOGITS) src = c->logits + ((size_t)(branch * S + slot) * W) * V;
+    else return HBSJD_EINVAL;
+    CK(cudaMemcpyAsync(host_dst, src, bytes, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return n;
+}
+
+int hbsjd_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
+    if (!c || !A || !W || !C || M < 1 || N < 1 || K < 1) return HBSJD_EINVAL;
+    int rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate) : gemm<float>(c, A, W, C, M, N, K, accumulate);
+    if (rc) return rc;
+    CK(cudaGetLastError());
+    return sync_counters(c);
+}
+
+}  // extern "C"

@@ -1,0 +1,89 @@
+// Launchers of the rollout kernels (internal to the library; the public boundary is include/hbsjd.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "common.cuh"
+
+namespace hbsjd {
+
+// Device-side rollout state and per-round slot tables.  A "slot" is the place of one image in the
+// physical batch of a forward: Full execution has one slot per image of the batch (finished images
+// get n = 0), Compact execution one slot per live image.  Token row of (branch, slot, i) =
+// (branch * S + slot) * W + i.
+struct State {
+    int B, T, V, D, Hh, dh, F, L, C;  // batch, tokens per image, vocab, dim, heads, head dim, ffn, layers, classes
+    int Bmax, Wmax;
+    int W, H;        // window (inputs per image per round), history offset
+    int nb;          // branches: 1, or 2 under classifier-free guidance
+    int32_t* cursor;   // [Bmax] committed tokens
+    int32_t* seq;      // [Bmax][T+1] tokens by 1-based position (committed, then drafts)
+    uint8_t* delta;    // [Bmax][T+1] draft carries a point-mass proposal
+    int32_t* qbase;    // [Bmax] cursor at the start of the previous round
+    int32_t* label;    // [Bmax]
+    int32_t* klen;     // [Bmax] prefix length
+    int32_t* pfill;    // [Bmax] prefill cursor
+    int32_t* slot_img; // [Bmax]
+    int32_t* slot_c;   // [Bmax] first sequence index of the slot's inputs
+    int32_t* slot_n;   // [Bmax] number of inputs (0: inactive slot)
+    int32_t* counters; // [8], see CNT_*
+    int32_t* m_last;   // [Bmax] tokens committed in the last round
+    int32_t* j_last;   // [Bmax] first-reject index of the last round (-1 none)
+};
+
+enum { CNT_LIVE = 0, CNT_COMMITTED = 1, CNT_REJECTS = 2, CNT_LIVE_SETUP = 3, CNT_SLOTS = 4, CNT_ERROR = 5,
+       CNT_SUM_KEYS = 6 /* sum over active slots of c+n */, CNT_SUM_N = 7 /* sum of n */ };
+
+struct AcceptArgs {
+    const float* logits;  // [nb][S][W][V]
+    float* pcur;          // [Bmax][Wmax][V] this round's probabilities (next round's proposals)
+    const float* pprev;   // [Bmax][Wmax][V]
+    uint8_t* flag;        // [Bmax][Wmax] 1 = draft accepted
+    int32_t* cand_rep;    // [Bmax][Wmax] replacement (or bonus) token candidate of position i
+    int32_t* cand_ref;    // [Bmax][Wmax] refreshed draft candidate of position i
+    int S;
+    float cfg_scale, temperature;
+    int top_k, greedy;
+    uint32_t seed_lo, seed_hi, round;
+};
+
+// ---- row operations (model_kernels.cu)
+void launch_setup(const State& st, int phase /*0 round, 1 prefill*/, int compact, cudaStream_t s);
+template <typename TA>
+void launch_embed(const State& st, int S, const TA* tok_emb, const TA* cls_emb, float* h, cudaStream_t s);
+template <typename TA>
+void launch_rmsnorm(const float* h, const TA* gain, TA* out, int M, int D, float eps, cudaStream_t s);
+template <typename TA>
+void launch_rope_kv(const State& st, int S, int layer, const float* qkv, const float* rope_cs, TA* q, KvView kv,
+                    cudaStream_t s);
+template <typename TA>
+void launch_attention_ref(const State& st, int S, int layer, const TA* q, KvView kv, TA* out, cudaStream_t s);
+template <typename TA>
+void launch_swiglu(const float* gu, TA* act, int M, int F, cudaStream_t s);
+template <typename TA>
+void launch_gemm_simt(const TA* A, const TA* W, float* C, int M, int N, int K, int accumulate, cudaStream_t s);
+
+// ---- tensor-core ragged attention, bf16, head size 64 (attention_mma.cu)
+bool attention_mma_supported(const State& st, const KvView& kv);
+void launch_attention_mma(const State& st, int S, int layer, const bf16* q, KvView kv, bf16* out, cudaStream_t s);
+
+// ---- state kernels (state_kernels.cu)
+void launch_init_state(const State& st, const int32_t* prefix_tokens, const int32_t* prefix_len,
+                       const int32_t* labels, cudaStream_t s);
+void launch_prefill_advance(const State& st, int S, cudaStream_t s);
+void launch_init_window(const State& st, uint32_t seed_lo, uint32_t seed_hi, cudaStream_t s);
+void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s);
+void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s);
+void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s);
+int accept_smem_bytes(int V);
+
+// ---- tcgen05 GEMM (gemm_tcgen05.cu)
+// C[M,N] fp32 (+)= A[M,K] bf16 . W[N,K]^T bf16.  force_bn: 0 = choose the tile width from the shape.
+// error_flag: device int set non-zero if a bounded pipeline wait gave up.  Returns 0, or a negative
+// code with a message in err.
+int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
+                     int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
+int gemm_tcgen05_tile_n(int M, int N);
+
+}  // namespace hbsjd

@@ -1,0 +1,460 @@
+// Rollout-state kernels: state init, prefill bookkeeping, initial history windows, and the fused
+// probability pipeline + SJD verification (Eq. 5; greedy Eq. 4) + commit + draft refresh.
+#include "internal.h"
+
+namespace hbsjd {
+
+// ------------------------------------------------------------------ state init (Sec. 4.2 "Independent rollout states")
+__global__ void k_init_state(State st, const int32_t* __restrict__ prefix_tokens,
+                             const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ labels) {
+    const int b = blockIdx.x;
+    const int k = prefix_len[b];
+    int32_t* seq = st.seq + (size_t)b * (st.T + 1);
+    uint8_t* dl = st.delta + (size_t)b * (st.T + 1);
+    for (int t = threadIdx.x; t <= st.T; t += blockDim.x) {
+        seq[t] = (t >= 1 && t <= k) ? prefix_tokens[(size_t)b * st.T + t - 1] : 0;
+        dl[t] = 0;
+    }
+    if (threadIdx.x == 0) {
+        st.cursor[b] = k;
+        st.klen[b] = k;
+        st.pfill[b] = 0;
+        st.qbase[b] = 0;
+        st.label[b] = labels[b];
+        st.m_last[b] = 0;
+        st.j_last[b] = -1;
+        if (b == 0)
+            for (int x = 0; x < 8; ++x)
+                if (x != CNT_ERROR) st.counters[x] = 0;
+    }
+}
+
+void launch_init_state(const State& st, const int32_t* prefix_tokens, const int32_t* prefix_len,
+                       const int32_t* labels, cudaStream_t s) {
+    k_init_state<<<st.B, 128, 0, s>>>(st, prefix_tokens, prefix_len, labels);
+}
+
+__global__ void k_prefill_advance(State st, int S) {
+    const int slot = blockIdx.x * blockDim.x + threadIdx.x;
+    if (slot >= S) return;
+    const int n = st.slot_n[slot];
+    if (n > 0) st.pfill[st.slot_img[slot]] = st.slot_c[slot] + n;
+}
+
+void launch_prefill_advance(const State& st, int S, cudaStream_t s) {
+    k_prefill_advance<<<(S + 127) / 128, 128, 0, s>>>(st, S);
+}
+
+// Initial window: every draft is the token H positions back, or a keyed uniform token where that
+// position does not exist; all are point-mass proposals.  Reserved round value 0xFFFFFFFF.
+__global__ void k_init_window(State st, uint32_t seed_lo, uint32_t seed_hi) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= st.B) return;
+    const int c = st.cursor[b];
+    if (c >= st.T) return;
+    int32_t* seq = st.seq + (size_t)b * (st.T + 1);
+    uint8_t* dl = st.delta + (size_t)b * (st.T + 1);
+    const int n = min(st.W, st.T - c);
+    for (int t = c + 1; t <= c + n - 1; ++t) {
+        const int src = t - st.H;
+        if (src >= 1) {
+            seq[t] = seq[src];
+        } else {
+            uint32_t w[4];
+            philox4x32_10((uint32_t)b, (uint32_t)t, 0xFFFFFFFFu, 0u, seed_lo, seed_hi, w);
+            seq[t] = (int32_t)(((uint64_t)w[3] * (uint64_t)st.V) >> 32);
+        }
+        dl[t] = 1;
+    }
+}
+
+void launch_init_window(const State& st, uint32_t seed_lo, uint32_t seed_hi, cudaStream_t s) {
+    k_init_window<<<(st.B + 63) / 64, 64, 0, s>>>(st, seed_lo, seed_hi);
+}
+
+__global__ void k_export_tokens(State st, int32_t* __restrict__ out) {
+    const int b = blockIdx.x;
+    for (int t = threadIdx.x; t < st.T; t += blockDim.x)
+        out[(size_t)b * st.T + t] = st.seq[(size_t)b * (st.T + 1) + t + 1];
+}
+
+void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s) {
+    k_export_tokens<<<st.B, 128, 0, s>>>(st, out);
+}
+
+// ------------------------------------------------------------------ probability pipeline + verification
+// One CTA per (slot, window position i).  The guided logits of the position live in shared memory:
+//   guided = l_u + s (l_c - l_u); / temperature; top-k threshold by radix select (ties kept);
+//   softmax -> p_i (written out: it is the proposal q of the drafts refreshed from it);
+//   accept test of draft z_{c+i+1}: u < min(1, p_i(z)/q(z))  (point-mass proposal: u < p_i(z))   [Eq. 5]
+//   candidates: refreshed draft ~ p_i (word 2); replacement ~ [p_i - q]+ (word 1) if rejected, or the
+//   bonus token ~ p_{n-1} (word 1) at the last position.
+// Sampling is fixed-point (weights floor(a 2^30), integer running sums), so the result does not depend
+// on the reduction order.  The per-image sequential part (first reject, commit, refresh) is k_commit.
+
+constexpr int ACC_THREADS = 512;
+constexpr int ACC_WARPS = ACC_THREADS / 32;
+
+struct AccShared {
+    unsigned int hist[ACC_WARPS][256];
+    float redf[ACC_WARPS];
+    unsigned long long redu[ACC_WARPS];
+    unsigned int sel_prefix, sel_k;
+    int result;
+    uint32_t words[4];
+    float bcast;
+};
+
+__device__ __forceinline__ unsigned int float_key(float x) {
+    const unsigned int u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__device__ __forceinline__ float block_max(float v, AccShared& sh) {
+    v = warp_max(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh.redf[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = sh.redf[0];
+#pragma unroll
+    for (int w = 1; w < ACC_WARPS; ++w) r = fmaxf(r, sh.redf[w]);
+    return r;
+}
+
+__device__ __forceinline__ float block_sum(float v, AccShared& sh) {
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sh.redf[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float r = 0.f;
+#pragma unroll
+    for (int w = 0; w < ACC_WARPS; ++w) r += sh.redf[w];
+    return r;
+}
+
+__device__ __forceinline__ unsigned int fixed_weight(float a) { return __float2uint_rd(a * 1073741824.0f); }
+
+// Fixed-point categorical sample over a[0..V) in shared memory (all threads call).  -1 if the total is 0.
+__device__ int block_sample(const float* a, int V, uint32_t word, AccShared& sh) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int seg = (((V + ACC_WARPS - 1) / ACC_WARPS) + 31) / 32 * 32;
+    const int base = wid * seg;
+    unsigned long long part = 0;
+    for (int it = 0; it < seg; it += 32) {
+        const int v = base + it + lane;
+        if (v < V) part += fixed_weight(a[v]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+    __syncthreads();
+    if (lane == 0) sh.redu[wid] = part;
+    if (threadIdx.x == 0) sh.result = -1;
+    __syncthreads();
+    unsigned long long S = 0;
+#pragma unroll
+    for (int w = 0; w < ACC_WARPS; ++w) S += sh.redu[w];
+    if (S == 0) return -1;
+    const unsigned long long target = ((unsigned long long)word * S) >> 32;
+    unsigned long long excl = 0;
+    for (int w = 0; w < wid; ++w) excl += sh.redu[w];
+    if (target >= excl && target < excl + sh.redu[wid]) {  // exactly one warp
+        unsigned long long run = excl;
+        for (int it = 0; it < seg; it += 32) {
+            const int v = base + it + lane;
+            unsigned long long x = (v < V) ? fixed_weight(a[v]) : 0ull;
+            unsigned long long incl = x;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const unsigned int hit = __ballot_sync(0xffffffffu, run + incl > target);
+            if (hit) {
+                if (lane == 0) sh.result = base + it + (__ffs(hit) - 1);
+                break;
+            }
+            run += __shfl_sync(0xffffffffu, incl, 31);
+        }
+    }
+    __syncthreads();
+    return sh.result;
+}
+
+__global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArgs a) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* g = (float*)smem_raw;  // [V]
+    AccShared& sh = *(AccShared*)(smem_raw + (size_t)st.V * sizeof(float));
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int i = blockIdx.x, slot = blockIdx.y;
+    const int n = st.slot_n[slot];
+    if (i >= n) return;
+    const int V = st.V;
+    const int img = st.slot_img[slot], c = st.slot_c[slot];
+    const int t = c + i + 1;  // token position this distribution decides
+    const float* lc = a.logits + ((size_t)slot * st.W + i) * V;
+    const float* lu = a.logits + ((size_t)(a.S + slot) * st.W + i) * V;
+    if (tid == 0) philox4x32_10((uint32_t)img, (uint32_t)t, a.round, 0u, a.seed_lo, a.seed_hi, sh.words);
+
+    // guided logits / temperature
+    const bool cfg = st.nb == 2;
+    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+        float4 x = *reinterpret_cast<const float4*>(lc + v);
+        if (cfg) {
+            const float4 y = *reinterpret_cast<const float4*>(lu + v);
+            x.x = __fadd_rn(y.x, __fmul_rn(a.cfg_scale, __fsub_rn(x.x, y.x)));
+            x.y = __fadd_rn(y.y, __fmul_rn(a.cfg_scale, __fsub_rn(x.y, y.y)));
+            x.z = __fadd_rn(y.z, __fmul_rn(a.cfg_scale, __fsub_rn(x.z, y.z)));
+            x.w = __fadd_rn(y.w, __fmul_rn(a.cfg_scale, __fsub_rn(x.w, y.w)));
+        }
+        x.x = __fdiv_rn(x.x, a.temperature);
+        x.y = __fdiv_rn(x.y, a.temperature);
+        x.z = __fdiv_rn(x.z, a.temperature);
+        x.w = __fdiv_rn(x.w, a.temperature);
+        *reinterpret_cast<float4*>(g + v) = x;
+    }
+    __syncthreads();
+
+    // top-k threshold: key of the k-th largest value, one byte per pass from the top
+    unsigned int theta = 0u;
+    if (a.top_k > 0 && a.top_k < V) {
+        if (tid == 0) {
+            sh.sel_prefix = 0u;
+            sh.sel_k = (unsigned int)a.top_k;
+        }
+        for (int pass = 0; pass < 4; ++pass) {
+            const int shift = 24 - 8 * pass;
+            const unsigned int mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+            for (int x = lane; x < 256; x += 32) sh.hist[wid][x] = 0u;
+            __syncthreads();
+            const unsigned int prefix = sh.sel_prefix;
+            for (int v = tid; v < V; v += ACC_THREADS) {
+                const unsigned int key = float_key(g[v]);
+                if ((key & mask) == prefix) atomicAdd(&sh.hist[wid][(key >> shift) & 255u], 1u);
+            }
+            __syncthreads();
+            if (wid == 0) {
+                // lane owns 8 consecutive bins (bins 8*lane .. 8*lane+7); scan from the top bin downwards
+                unsigned int cnt[8], tot = 0;
+#pragma unroll
+                for (int x = 0; x < 8; ++x) {
+                    unsigned int s = 0;
+                    for (int w = 0; w < ACC_WARPS; ++w) s += sh.hist[w][lane * 8 + x];
+                    cnt[x] = s;
+                    tot += s;
+                }
+                // suffix sum over lanes: above = elements in bins of higher lanes
+                unsigned int incl = tot;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned int tt = __shfl_down_sync(0xffffffffu, incl, o);
+                    if (lane + o < 32) incl += tt;
+                }
+                unsigned int above = incl - tot;
+                const unsigned int k = sh.sel_k;
+                if (above < k && k <= above + tot) {  // exactly one lane
+#pragma unroll
+                    for (int x = 7; x >= 0; --x) {
+                        if (above < k && k <= above + cnt[x]) {
+                            sh.sel_prefix = prefix | ((unsigned int)(lane * 8 + x) << shift);
+                            sh.sel_k = k - above;
+                            above = 0xFFFFFFFFu;  // done
+                        } else if (above != 0xFFFFFFFFu) {
+                            above += cnt[x];
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+        }
+        theta = sh.sel_prefix;
+    }
+
+    // softmax over the kept entries
+    float mx = -INFINITY;
+    for (int v = tid; v < V; v += ACC_THREADS) {
+        const float x = g[v];
+        if (float_key(x) >= theta) mx = fmaxf(mx, x);
+    }
+    mx = block_max(mx, sh);
+    float part = 0.f;
+    for (int v = tid; v < V; v += ACC_THREADS) {
+        const float x = g[v];
+        const float e = float_key(x) >= theta ? expf(x - mx) : 0.f;
+        g[v] = e;
+        part += e;
+    }
+    const float den = block_sum(part, sh);
+    float* pout = a.pcur + ((size_t)img * st.Wmax + i) * V;
+    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+        float4 e = *reinterpret_cast<float4*>(g + v);
+        e.x = __fdiv_rn(e.x, den);
+        e.y = __fdiv_rn(e.y, den);
+        e.z = __fdiv_rn(e.z, den);
+        e.w = __fdiv_rn(e.w, den);
+        *reinterpret_cast<float4*>(g + v) = e;
+        *reinterpret_cast<float4*>(pout + v) = e;
+    }
+    __syncthreads();
+
+    const size_t oidx = (size_t)img * st.Wmax + i;
+    const bool last = (i == n - 1);
+    const int z = last ? 0 : st.seq[(size_t)img * (st.T + 1) + t];
+    const bool is_delta = last ? false : (st.delta[(size_t)img * (st.T + 1) + t] != 0);
+    const int qi = (last || is_delta) ? 0 : (t - st.qbase[img] - 1);  // row of the previous round's probabilities
+    const float* qrow = a.pprev + ((size_t)img * st.Wmax + qi) * V;
+
+    if (a.greedy) {
+        // argmax, lowest index on ties
+        unsigned long long best = 0ull;
+        for (int v = tid; v < V; v += ACC_THREADS) {
+            const unsigned long long key =
+                ((unsigned long long)__float_as_uint(g[v]) << 32) | (unsigned long long)(0xFFFFFFFFu - (unsigned)v);
+            best = key > best ? key : best;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+            best = other > best ? other : best;
+        }
+        __syncthreads();
+        if (lane == 0) sh.redu[wid] = best;
+        __syncthreads();
+        if (tid == 0) {
+            unsigned long long b2 = sh.redu[0];
+            for (int w = 1; w < ACC_WARPS; ++w) b2 = sh.redu[w] > b2 ? sh.redu[w] : b2;
+            const int am = (int)(0xFFFFFFFFu - (unsigned)(b2 & 0xFFFFFFFFull));
+            a.cand_rep[oidx] = am;
+            a.cand_ref[oidx] = am;
+            a.flag[oidx] = (!last && z == am) ? 1 : 0;
+        }
+        return;
+    }
+
+    // accept test (Eq. 5)
+    bool accept = true;
+    if (!last) {
+        if (tid == 0) {
+            const float pz = g[z];
+            float alpha;
+            if (is_delta) alpha = pz;
+            else alpha = fminf(1.0f, __fdiv_rn(pz, qrow[z]));
+            const float u = (float)(sh.words[0] >> 8) * (1.0f / 16777216.0f);
+            sh.bcast = (u < alpha) ? 1.f : 0.f;
+            a.flag[oidx] = (u < alpha) ? 1 : 0;
+        }
+        __syncthreads();
+        accept = sh.bcast != 0.f;
+    }
+    const uint32_t w1 = sh.words[1], w2 = sh.words[2];
+
+    // refreshed draft candidate ~ p_i
+    const int ref = block_sample(g, V, w2, sh);
+    int rep = -1;
+    if (last) {
+        rep = block_sample(g, V, w1, sh);  // bonus token ~ p_{n-1}
+    } else if (!accept) {
+        // residual [p - q]+ (point-mass proposal: p with z removed), overwriting p in shared memory
+        if (is_delta) {
+            if (tid == 0) g[z] = 0.f;
+        } else {
+            for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+                float4 p4 = *reinterpret_cast<float4*>(g + v);
+                const float4 q4 = *reinterpret_cast<const float4*>(qrow + v);
+                p4.x = fmaxf(__fsub_rn(p4.x, q4.x), 0.f);
+                p4.y = fmaxf(__fsub_rn(p4.y, q4.y), 0.f);
+                p4.z = fmaxf(__fsub_rn(p4.z, q4.z), 0.f);
+                p4.w = fmaxf(__fsub_rn(p4.w, q4.w), 0.f);
+                *reinterpret_cast<float4*>(g + v) = p4;
+            }
+        }
+        __syncthreads();
+        rep = block_sample(g, V, w1, sh);
+        if (rep < 0) {  // empty residual: sample p_i itself with the same word
+            __syncthreads();
+            for (int v = tid * 4; v < V; v += ACC_THREADS * 4)
+                *reinterpret_cast<float4*>(g + v) = *reinterpret_cast<const float4*>(pout + v);
+            __syncthreads();
+            rep = block_sample(g, V, w1, sh);
+        }
+    }
+    if (tid == 0) {
+        a.cand_ref[oidx] = ref;
+        a.cand_rep[oidx] = rep;
+    }
+}
+
+int accept_smem_bytes(int V) { return V * (int)sizeof(float) + (int)sizeof(AccShared); }
+
+void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
+    static int configured_bytes = 0;
+    const int bytes = accept_smem_bytes(st.V);
+    if (bytes > configured_bytes) {
+        cudaFuncSetAttribute(k_prob_accept, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        configured_bytes = bytes;
+    }
+    dim3 grid(st.W, a.S);
+    k_prob_accept<<<grid, ACC_THREADS, accept_smem_bytes(st.V), s>>>(st, a);
+}
+
+// ------------------------------------------------------------------ commit + refresh (one warp per slot)
+// First reject by ballot over the accept flags; lane 0 commits the accepted prefix plus the replacement
+// (or bonus) token, advances the cursor -- the KV commit is this cursor move: entries at and after the
+// new cursor are recomputed by the next forward (Sec. 4.2 "Independent progress") -- and rebuilds the window.
+__global__ void k_commit(State st, AcceptArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (slot >= a.S) return;
+    const int n = st.slot_n[slot];
+    if (n == 0) return;
+    const int img = st.slot_img[slot], c = st.slot_c[slot];
+    int j = -1;
+    for (int base = 0; base < n - 1; base += 32) {
+        const int i = base + lane;
+        const bool rej = (i < n - 1) && (a.flag[(size_t)img * st.Wmax + i] == 0);
+        const unsigned int b = __ballot_sync(0xffffffffu, rej);
+        if (b) {
+            j = base + __ffs(b) - 1;
+            break;
+        }
+    }
+    if (lane != 0) return;
+    int32_t* seq = st.seq + (size_t)img * (st.T + 1);
+    uint8_t* dl = st.delta + (size_t)img * (st.T + 1);
+    const int m = j >= 0 ? j + 1 : n;
+    const int tok = a.cand_rep[(size_t)img * st.Wmax + (m - 1)];
+    seq[c + m] = tok;
+    dl[c + m] = 0;
+    const int c2 = c + m;
+    st.cursor[img] = c2;
+    st.qbase[img] = c;
+    st.m_last[img] = m;
+    st.j_last[img] = j;
+    if (c2 < st.T) {
+        const int n2 = min(st.W, st.T - c2);
+        for (int t = c2 + 1; t <= c2 + n2 - 1; ++t) {
+            if (t <= c + n) {
+                seq[t] = a.cand_ref[(size_t)img * st.Wmax + (t - c - 1)];
+                dl[t] = 0;
+            } else {
+                const int src = t - st.H;
+                if (src >= 1) {
+                    seq[t] = seq[src];
+                } else {
+                    uint32_t w[4];
+                    philox4x32_10((uint32_t)img, (uint32_t)t, a.round, 0u, a.seed_lo, a.seed_hi, w);
+                    seq[t] = (int32_t)(((uint64_t)w[3] * (uint64_t)st.V) >> 32);
+                }
+                dl[t] = 1;
+            }
+        }
+        atomicAdd(&st.counters[CNT_LIVE], 1);
+    }
+    atomicAdd(&st.counters[CNT_COMMITTED], m);
+    if (j >= 0) atomicAdd(&st.counters[CNT_REJECTS], 1);
+}
+
+void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s) {
+    k_commit<<<(a.S + 3) / 4, 128, 0, s>>>(st, a);
+}
+
+}  // namespace hbsjd

@@ -93,6 +93,8 @@ WORKLOADS = {
     # small shapes for tests: same structure, sizes the CPU oracle finishes quickly
     "tiny_bf16": Workload("tiny_bf16", _shape(2, 128, 2, 384, 512, 8, 10, "bf16"), 6, 8, 3.0, 50, 1.0, 8,
                           ("uniform", 0, 20)),
+    "small_bf16": Workload("small_bf16", ModelShape(2, 256, 4, 512, 1024, 12, 12, 10, "bf16"), 6, 32, 2.0, 100, 1.0,
+                           12, ("uniform", 0, 100)),
     "micro": Workload("micro", _shape(1, 16, 1, 32, 6, 2, 3, "fp32"), 1, 2, 1.0, 0, 1.0, 2, ("const", 0)),
 }
 

@@ -1,0 +1,155 @@
+"""Helpers of the GPU parity tests: contexts on the CUDA library, oracle rollouts, lockstep comparison."""
+import numpy as np
+
+from oracle import oracle as O
+from paper_2608_18183_b200 import binding, synth
+
+_weights = {}
+
+
+def weights_for(w):
+    key = (w.shape, w.weight_seed)
+    if key not in _weights:
+        _weights[key] = synth.make_weights(w.shape, w.weight_seed)
+    return _weights[key]
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def gpu_params(w, seed, **kw):
+    d = dict(window=w.window, history_offset=w.history_offset, cfg_scale=w.cfg_scale, temperature=w.temperature,
+             top_k=w.top_k, seed=seed)
+    d.update(kw)
+    return binding.make_params(**d)
+
+
+def orc_params(w, seed, greedy=False, window=None, history=None, exec_mode=0, gamma=0):
+    return O.make_params(window or w.window, history or w.history_offset, cfg_scale=w.cfg_scale,
+                         temperature=w.temperature, top_k=w.top_k, greedy=greedy, exec_mode=exec_mode, gamma=gamma,
+                         seed=seed)
+
+
+def residual_cdf_distance(p, q, is_delta, z, word):
+    """Distance (as a fraction of the total mass) of the fixed-point target of `word` from the
+    nearest bin edge of the replacement distribution."""
+    if q is None:
+        a = p.astype(np.float64).copy()
+    elif is_delta:
+        a = p.astype(np.float64).copy()
+        a[z] = 0
+    else:
+        a = np.maximum(p.astype(np.float32) - q.astype(np.float32), 0).astype(np.float64)
+    if a.sum() == 0:
+        a = p.astype(np.float64)
+    cdf = np.cumsum(a) / a.sum()
+    x = word / 2.0 ** 32
+    return float(np.min(np.abs(cdf - x)))
+
+
+def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, max_rounds=None, gpu_batch=None,
+             check_replay=True):
+    """Runs the oracle and the GPU round by round, the GPU state re-synchronised to the oracle's before
+    each round.  `image_ids` restricts the oracle to a subset of the GPU batch.  Returns a report dict."""
+    ids = list(range(len(k))) if image_ids is None else list(image_ids)
+    V, T, W = w.shape.vocab, w.shape.T, w.window
+    P = orc_params(w, seed, greedy=greedy)
+    orc = O.Rollout(model, toks[ids], k[ids], lab[ids], P, image_ids=ids)
+    gp = gpu_params(w, seed, verify_mode=1 if greedy else 0, max_rounds=0, exec_mode=binding.EXEC_FULL)
+    ctx.hbsjd_rollout(dev(toks), dev(k), dev(lab), gp)
+    g_r, g_cur, g_seq, g_dl, g_qb = ctx.hbsjd_get_state()
+    o_r, o_cur, o_seq, o_dl, o_qb = orc.state()
+    # the initial windows are integer work: bit-exact
+    assert g_r == 0 and o_r == 0
+    np.testing.assert_array_equal(g_cur[ids], o_cur)
+    np.testing.assert_array_equal(g_seq[ids], o_seq)
+    np.testing.assert_array_equal(g_dl[ids], o_dl)
+    rep = dict(tokens=0, same=0, flips=[], rounds=0, max_logit_err=0.0, max_p_err=0.0, replay_mismatch=0,
+               m_gpu=0, m_orc=0, logit_std=0.0)
+    qprev = {b: np.zeros((W, V), dtype=np.float32) for b in ids}
+    full_state = list(ctx.hbsjd_get_state())
+    while orc.live() and (max_rounds is None or rep["rounds"] < max_rounds):
+        o_r, o_cur, o_seq, o_dl, o_qb = orc.state()
+        _, cur, seq, dl, qb = [x.copy() if hasattr(x, "copy") else x for x in full_state]
+        cur[ids], seq[ids], dl[ids], qb[ids] = o_cur, o_seq, o_dl, o_qb
+        # images outside the subset are parked as finished
+        others = [b for b in range(len(k)) if b not in ids]
+        cur[others] = T
+        ctx.hbsjd_set_state(o_r, cur, seq, dl, qb)
+        ctx.hbsjd_round()
+        g_r, g_cur, g_seq, g_dl, g_qb = ctx.hbsjd_get_state()
+        full_state = [g_r, g_cur, g_seq, g_dl, g_qb]
+        oq = {x: orc.last_probs(x) for x in range(len(ids))}  # the oracle's proposals of this round
+        _, om, oj = orc.round()
+        n_r, n_cur, n_seq, n_dl, n_qb = orc.state()
+        for x, b in enumerate(ids):
+            c = int(o_cur[x])
+            if c >= T:
+                continue
+            n = min(W, T - c)
+            gl = ctx.hbsjd_debug_read(binding.DBG_LOGITS, 2 * b)
+            ol = orc.last_logits(x, 0)
+            rep["max_logit_err"] = max(rep["max_logit_err"], float(np.abs(gl - ol).max()))
+            rep["logit_std"] = max(rep["logit_std"], float(ol.std()))
+            if w.cfg_scale != 1.0:
+                glu = ctx.hbsjd_debug_read(binding.DBG_LOGITS, 2 * b + 1)
+                rep["max_logit_err"] = max(rep["max_logit_err"], float(np.abs(glu - orc.last_logits(x, 1)).max()))
+            gp_ = ctx.hbsjd_debug_read(binding.DBG_PROBS, b)
+            op_ = orc.last_probs(x)
+            assert gp_.shape == (n, V)
+            # probabilities from the GPU's own logits through the oracle's pipeline
+            pl = np.stack([O.probs(gl[i], glu[i] if w.cfg_scale != 1.0 else None, s=w.cfg_scale, tau=w.temperature,
+                                   k=w.top_k) for i in range(n)])
+            rep["max_p_err"] = max(rep["max_p_err"], float((np.abs(gp_ - pl) - 1e-4 * pl).max()))
+            if check_replay:
+                # verify / commit / refresh replayed by the oracle on the GPU's probabilities: bit-exact
+                s2, d2 = o_seq[x].copy(), o_dl[x].copy()
+                nc, mm, jj = O.replay_round(V, T, W, w.history_offset, greedy, seed, b, o_r, c, s2, d2, gp_,
+                                            qprev[b], int(o_qb[x]))
+                ok = nc == g_cur[b] and np.array_equal(s2[:nc + W], g_seq[b][:nc + W]) and np.array_equal(
+                    d2[nc + 1:nc + W], g_dl[b][nc + 1:nc + W])
+                rep["replay_mismatch"] += 0 if ok else 1
+            # committed tokens against the oracle's own round
+            m_o, m_g = int(n_cur[x]) - c, int(g_cur[b]) - c
+            rep["m_gpu"] += m_g
+            rep["m_orc"] += m_o
+            rep["tokens"] += m_o
+            same = 0
+            for t in range(c + 1, c + m_o + 1):
+                if t <= c + m_g and g_seq[b][t] == n_seq[x][t]:
+                    same += 1
+                else:
+                    break
+            rep["same"] += same
+            if same != m_o or m_g != m_o:
+                # classify the first differing decision
+                i = same  # window position whose decision differs
+                t = c + i + 1
+                words = O.philox([b, t, o_r, 0], [seed & 0xffffffff, seed >> 32])
+                info = dict(image=b, round=o_r, pos=t, m_gpu=m_g, m_orc=m_o)
+                if greedy:
+                    # the GPU's argmax at this position is the token it committed there
+                    if t <= c + m_g:
+                        a_g, a_o = int(g_seq[b][t]), int(np.argmax(op_[i]))
+                        info["argmax_gap"] = 1.0 - float(op_[i][a_g]) / float(op_[i][a_o])
+                if not greedy:
+                    u = float(words[0] >> 8) / 2 ** 24
+                    z = int(o_seq[x][t])
+                    if i < n - 1:
+                        if o_dl[x][t]:
+                            alpha, qrow = float(op_[i][z]), None
+                        else:
+                            qrow = oq[x][t - int(o_qb[x]) - 1]
+                            alpha = min(1.0, float(op_[i][z]) / float(qrow[z]))
+                        info["u_minus_alpha"] = abs(u - alpha)
+                        info["cdf_dist"] = residual_cdf_distance(op_[i], qrow, bool(o_dl[x][t]), z, int(words[1]))
+                    else:
+                        info["u_minus_alpha"] = None
+                        info["cdf_dist"] = residual_cdf_distance(op_[i], None, False, 0, int(words[1]))
+                rep["flips"].append(info)
+            qprev[b] = gp_
+        rep["rounds"] += 1
+    return rep
+
