@@ -25,7 +25,6 @@ struct hbsjd_ctx {
     hbsjd_model_desc d;
     int T, dh, Bmax, Wmax;
     bool bf16_model;
-    bool simt_gemm;      // debugging: run the bf16 GEMMs on CUDA cores
     bool ref_attention;  // debugging: run the one-warp-per-row attention kernel
     cudaStream_t stream;
     // weights
@@ -148,11 +147,6 @@ template <>
 int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
     c->launches++;
     const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
-    if (c->simt_gemm) {
-        launch_gemm_simt<bf16>((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, c->stream);
-        prof_end(c, ps);
-        return 0;
-    }
     const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, 0,
                                     c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err));
     prof_end(c, ps);
@@ -172,8 +166,19 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
         const LayerW& w = c->layers[l];
         int rc;
         launch_rmsnorm<TA>(c->h, (const TA*)w.g_attn, (TA*)c->a, M, D, c->d.rms_eps, s);
-        if ((rc = gemm<TA>(c, c->a, w.w_qkv, c->qkv, M, 3 * D, D, 0))) return rc;
-        launch_rope_kv<TA>(st, S, l, c->qkv, c->rope_cs, (TA*)c->q, kv, s);
+        if constexpr (std::is_same<TA, bf16>::value) {
+            // QKV projection with RoPE and the paged KV write in its epilogue
+            const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D);
+            rc = gemm_tcgen05_qkv((const bf16*)c->a, (const bf16*)w.w_qkv, (bf16*)c->q, st, S, l, c->rope_cs, kv,
+                                  c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
+            prof_end(c, ps);
+            if (rc) return rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
+            c->launches += 2;
+        } else {
+            if ((rc = gemm<TA>(c, c->a, w.w_qkv, c->qkv, M, 3 * D, D, 0))) return rc;
+            launch_rope_kv<TA>(st, S, l, c->qkv, c->rope_cs, (TA*)c->q, kv, s);
+            c->launches += 2;
+        }
         {
             const int ps = prof_begin(c, HBSJD_PROF_ATTENTION, 0.0);
             if constexpr (std::is_same<TA, bf16>::value) {
@@ -185,13 +190,25 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
                 launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
             }
             prof_end(c, ps);
+            c->launches++;
         }
         if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1))) return rc;
         launch_rmsnorm<TA>(c->h, (const TA*)w.g_ffn, (TA*)c->a, M, D, c->d.rms_eps, s);
-        if ((rc = gemm<TA>(c, c->a, w.w_13, c->gu, M, 2 * F, D, 0))) return rc;
-        launch_swiglu<TA>(c->gu, (TA*)c->act, M, F, s);
+        c->launches++;
+        if constexpr (std::is_same<TA, bf16>::value) {
+            // gate/up projection with SwiGLU in its epilogue (gate and up rows interleaved at load time)
+            const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D);
+            rc = gemm_tcgen05_swiglu((const bf16*)c->a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D,
+                                     c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
+            prof_end(c, ps);
+            if (rc) return rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
+            c->launches++;
+        } else {
+            if ((rc = gemm<TA>(c, c->a, w.w_13, c->gu, M, 2 * F, D, 0))) return rc;
+            launch_swiglu<TA>(c->gu, (TA*)c->act, M, F, s);
+            c->launches++;
+        }
         if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1))) return rc;
-        c->launches += 5;
     }
     if (want_logits) {
         launch_rmsnorm<TA>(c->h, (const TA*)c->g_out, (TA*)c->a, M, D, c->d.rms_eps, s);
@@ -334,6 +351,20 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
     }
     CK(cudaMalloc((void**)&c->w_img, off));
     CK(cudaMemcpyAsync(c->w_img, weights, off, cudaMemcpyHostToDevice, c->stream));
+    if (c->bf16_model) {
+        // the SwiGLU epilogue wants gate row f and up row f next to each other: rows (2f, 2f+1)
+        std::vector<uint16_t> tmp(2 * F * D);
+        for (size_t l = 0; l < L; ++l) {
+            const uint16_t* src = (const uint16_t*)((const unsigned char*)weights + lo[l * 6 + 4]);
+            for (size_t f = 0; f < F; ++f) {
+                memcpy(&tmp[(2 * f) * D], src + f * D, D * 2);
+                memcpy(&tmp[(2 * f + 1) * D], src + (F + f) * D, D * 2);
+            }
+            CK(cudaMemcpyAsync(c->w_img + lo[l * 6 + 4], tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice,
+                               c->stream));
+            CK(cudaStreamSynchronize(c->stream));
+        }
+    }
     c->tok_emb = c->w_img + o_tok;
     c->cls_emb = c->w_img + o_cls;
     c->g_out = c->w_img + o_gout;
@@ -410,8 +441,9 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
     // activations for the largest forward: 2 branches x max_batch slots x max_window inputs
     const size_t Mmax = 2 * Bm * Wm;
     unsigned char *a, *q, *o, *act;
-    if ((rc = dev_alloc(c, &c->h, Mmax * D)) || (rc = dev_alloc(c, &c->qkv, Mmax * 3 * D)) ||
-        (rc = dev_alloc(c, &c->gu, Mmax * 2 * F)) || (rc = dev_alloc(c, &c->logits, Mmax * V)) ||
+    const size_t f32_only = c->bf16_model ? 0 : 1;  // fp32 GEMM outputs the fused bf16 epilogues never materialise
+    if ((rc = dev_alloc(c, &c->h, Mmax * D)) || (rc = dev_alloc(c, &c->qkv, f32_only * Mmax * 3 * D)) ||
+        (rc = dev_alloc(c, &c->gu, f32_only * Mmax * 2 * F)) || (rc = dev_alloc(c, &c->logits, Mmax * V)) ||
         (rc = dev_alloc(c, &a, Mmax * D * es)) || (rc = dev_alloc(c, &q, Mmax * D * es)) ||
         (rc = dev_alloc(c, &o, Mmax * D * es)) || (rc = dev_alloc(c, &act, Mmax * F * es)))
         return rc;
@@ -467,7 +499,8 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     const int dh = m->dim / m->n_heads;
     if (dh != 16 && dh != 32 && dh != 64 && dh != 128) return HBSJD_EINVAL;
     if (m->dim % 16 || m->ffn_hidden % 16) return HBSJD_EINVAL;
-    if (m->dtype == HBSJD_DTYPE_BF16 && (m->dim % 64 || m->ffn_hidden % 64 || m->vocab % 64)) return HBSJD_EINVAL;
+    if (m->dtype == HBSJD_DTYPE_BF16 && (m->dim % 64 || m->ffn_hidden % 64 || m->vocab % 64 || dh < 32))
+        return HBSJD_EINVAL;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return HBSJD_ECUDA;
     hbsjd_ctx* c = new (std::nothrow) hbsjd_ctx();
@@ -479,8 +512,6 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     c->Bmax = max_batch;
     c->Wmax = max_window;
     c->bf16_model = m->dtype == HBSJD_DTYPE_BF16;
-    const char* g = getenv("HBSJD_GEMM");
-    c->simt_gemm = g && strcmp(g, "simt") == 0;
     const char* at = getenv("HBSJD_ATTENTION");
     c->ref_attention = at && strcmp(at, "ref") == 0;
     c->stream = (cudaStream_t)cuda_stream;

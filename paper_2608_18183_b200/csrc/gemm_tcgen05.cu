@@ -1,17 +1,26 @@
-// bf16 decoder GEMM on the 5th-generation tensor cores: C[M,N] fp32 (+)= A[M,K] . W[N,K]^T.
+// bf16 decoder GEMMs on the 5th-generation tensor cores: acc[M,N] = A[M,K] . W[N,K]^T with fused epilogues.
 //
-// Both operands are K-major (activations row-major [M,K], weights row-major [N,K]), so each CTA
-// streams 128 x 64 (A) and BN x 64 (W) bf16 tiles through a TMA -> shared-memory ring
-// (128-byte swizzle), one elected thread issues tcgen05.mma (M=128, N=BN, K=16) into a TMEM
-// accumulator, and four warps read the accumulator back with tcgen05.ld for the epilogue.
-// The K loop is fixed (no split-K), so an output element's rounding does not depend on M or on
-// which rows share its tile: Full and Compact execution give identical bits.
+// Both operands are K-major (activations row-major [M,K], weights row-major [N,K]).  The kernel is
+// persistent and warp-specialised: one CTA per SM walks a static list of 128 x BN output tiles;
+//   warp 0 (one lane)  TMA producer: 128 x 64 (A) and BN x 64 (W) bf16 tiles, 128-byte swizzle, STAGES-deep ring
+//   warp 1 (one lane)  issues tcgen05.mma (M = 128, N = BN, K = 16) into one of two TMEM accumulators
+//   warps 2..5         epilogue: tcgen05.ld of the finished accumulator while the next tile's main loop runs
+// BN = 256 keeps the shared-memory operand traffic per MMA below the 128 B/clk the SM can supply.
+// The K loop is fixed (no split-K), so an output element's rounding does not depend on M or on which rows
+// share its tile: Full and Compact execution give identical bits.
 //
-// Every mbarrier wait is bounded: after the limit the kernel raises the error flag, drains, frees its
-// TMEM and returns.  No cluster launch, no multicast.
+// Epilogues:  STORE  C fp32 = acc           (LM head -> logits)
+//             ADD    C fp32 += acc          (attention-out and FFN-down projections into the residual stream)
+//             SWIGLU out bf16[M, N/2] = silu(acc[2f]) * acc[2f+1]   (gate/up rows interleaved at load time)
+//             QKV    2D RoPE on q and k, bf16 q[M, D], k and v written to the row's KV pages
+//
+// Every mbarrier wait is bounded (about a second): after the limit the kernel raises the error flag, all
+// roles leave their loops, TMEM is freed and the kernel returns.  No cluster launch, no multicast.
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstdlib>
+#include <cstring>
 
 #include "internal.h"
 
@@ -21,6 +30,21 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
+constexpr int NUM_THREADS = 192;
+
+enum { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
+
+struct GemmArgs {
+    float* C;        // STORE / ADD
+    bf16* out;       // SWIGLU: [M, N/2];  QKV: q [M, D]
+    int M, N, K;
+    int32_t* error_flag;
+    // QKV epilogue
+    State st;
+    int S, layer;
+    const float* rope_cs;  // [T][dh/2][2]
+    KvView kv;
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -29,6 +53,9 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
     uint32_t ok;
@@ -46,13 +73,14 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait (about one second).  Returns false when it gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait (about one second).  Returns false when it gave up or another role raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort) {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
-        for (int it = 0; it < 256; ++it)
+        for (int it = 0; it < 128; ++it)
             if (mbar_try(bar, parity)) return true;
+        if (*abort) return false;
         if (globaltimer_ns() - t0 > 1000000000ull) return false;
     }
 }
@@ -91,42 +119,75 @@ __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t 
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t r[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
 
 template <int BN>
 struct Cfg {
-    static constexpr int STAGES = BN >= 256 ? 4 : (BN == 128 ? 3 : 4);
+    static constexpr int STAGES = 4;
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int TMEM_COLS = BN < 32 ? 32 : BN;
-    static constexpr int SMEM = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;  // two accumulators
+    static constexpr int STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffers x (32 rows x 128 bytes)
+    static constexpr int SMEM = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
-template <int BN>
-__global__ void __launch_bounds__(128) k_gemm_tcgen05(const __grid_constant__ CUtensorMap map_a,
-                                                      const __grid_constant__ CUtensorMap map_w,
-                                                      float* __restrict__ C, int M, int N, int K, int accumulate,
-                                                      int32_t* __restrict__ error_flag) {
+// Per-row context of the QKV epilogue: where the token row's q / k / v go.
+struct RowDst {
+    bool valid;
+    int s;        // sequence index (RoPE position)
+    size_t kvoff; // element offset of the row's K/V vector in the page pool
+};
+
+template <int BN, int EPI>
+__global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_constant__ CUtensorMap map_a,
+                                                              const __grid_constant__ CUtensorMap map_w,
+                                                              const __grid_constant__ CUtensorMap map_c,
+                                                              const GemmArgs g) {
     using cfg = Cfg<BN>;
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t tiles = (raw + 1023u) & ~1023u;            // 1024-byte aligned tile ring
-    const uint32_t bars = tiles + cfg::STAGES * cfg::STAGE_BYTES;  // full[STAGES], empty[STAGES], accum, tmem slot
+    const uint32_t tiles = (raw + 1023u) & ~1023u;  // 1024-byte aligned tile ring
+    const uint32_t staging = tiles + cfg::STAGES * cfg::STAGE_BYTES;  // 1024-byte aligned
+    const uint32_t bars = staging + cfg::STAGING_BYTES;
     unsigned char* bars_ptr = smem_raw + (bars - raw);
-    const uint32_t full0 = bars, empty0 = bars + 8 * cfg::STAGES, accum_bar = bars + 16 * cfg::STAGES;
-    volatile uint32_t* tmem_slot = (volatile uint32_t*)(bars_ptr + 16 * cfg::STAGES + 8);
+    // full[STAGES], empty[STAGES], acc_full[2], acc_empty[2], tmem slot, abort flag
+    const uint32_t full0 = bars, empty0 = bars + 8 * cfg::STAGES;
+    const uint32_t accf0 = bars + 16 * cfg::STAGES, acce0 = accf0 + 16;
+    volatile uint32_t* tmem_slot = (volatile uint32_t*)(bars_ptr + 16 * cfg::STAGES + 32);
     volatile uint32_t* abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM;
-    const int num_kb = K / BK;
+    const int M = g.M, N = g.N;
+    const int num_kb = g.K / BK;
+    const int tiles_n = N / BN, tiles_m = (M + BM - 1) / BM;
+    const int num_tiles = tiles_n * tiles_m;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < cfg::STAGES; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, 1);
         }
-        mbar_init(accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(accf0 + 8 * b, 1);
+            mbar_init(acce0 + 8 * b, 4);  // one arrival per epilogue warp
+        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -142,88 +203,182 @@ __global__ void __launch_bounds__(128) k_gemm_tcgen05(const __grid_constant__ CU
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == 0 && lane == 0) {
-        // ---- TMA producer
-        for (int kb = 0; kb < num_kb; ++kb) {
-            const int s = kb % cfg::STAGES;
-            if (kb >= cfg::STAGES) {
-                if (!mbar_wait(empty0 + 8 * s, ((kb / cfg::STAGES) - 1) & 1)) {
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t kc = 0;
+            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
+                const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+                bool ok = true;
+                for (int kb = 0; kb < num_kb; ++kb, ++kc) {
+                    const uint32_t s = kc % cfg::STAGES, ph = (kc / cfg::STAGES) & 1u;
+                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
+                        *abort_flag = 1;
+                        atomicExch(g.error_flag, 1);
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t a_dst = tiles + s * cfg::STAGE_BYTES;
+                    mbar_expect_tx(full0 + 8 * s, cfg::STAGE_BYTES);
+                    tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
+                    tma_load_2d(a_dst + cfg::A_BYTES, &map_w, kb * BK, n0, full0 + 8 * s);
+                }
+                if (!ok) break;
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc(BN);
+            uint32_t kc = 0, j = 0;
+            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++j) {
+                const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
+                bool ok = mbar_wait(acce0 + 8 * buf, aph ^ 1u, abort_flag);  // epilogue drained this accumulator
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + buf * BN;
+                for (int kb = 0; kb < num_kb && ok; ++kb, ++kc) {
+                    const uint32_t s = kc % cfg::STAGES, ph = (kc / cfg::STAGES) & 1u;
+                    if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_src = tiles + s * cfg::STAGE_BYTES;
+                    const uint32_t b_src = a_src + cfg::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_f16(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc,
+                                 (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(empty0 + 8 * s);  // frees the stage once these MMAs have read it
+                }
+                if (!ok) {
                     *abort_flag = 1;
-                    atomicExch(error_flag, 1);
+                    atomicExch(g.error_flag, 2);
                     break;
                 }
+                umma_commit(accf0 + 8 * buf);  // accumulator complete
             }
-            const uint32_t a_dst = tiles + s * cfg::STAGE_BYTES;
-            const uint32_t b_dst = a_dst + cfg::A_BYTES;
-            mbar_expect_tx(full0 + 8 * s, cfg::STAGE_BYTES);
-            tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
-            tma_load_2d(b_dst, &map_w, kb * BK, n0, full0 + 8 * s);
         }
-    } else if (warp == 1 && lane == 0) {
-        // ---- MMA issuer
-        constexpr uint32_t idesc = umma_idesc(BN);
-        bool ok = true;
-        for (int kb = 0; kb < num_kb && ok; ++kb) {
-            const int s = kb % cfg::STAGES;
-            if (!mbar_wait(full0 + 8 * s, (kb / cfg::STAGES) & 1)) {
-                *abort_flag = 1;
-                atomicExch(error_flag, 2);
-                ok = false;
+    } else {
+        // ---------------------------------------------------------------- epilogue warps 2..5
+        const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter+31 belong to this warp
+        uint32_t j = 0, nchunk = 0;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++j) {
+            const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+            const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
+            if (!mbar_wait(accf0 + 8 * buf, aph, abort_flag)) {
+                if (lane == 0) {
+                    *abort_flag = 1;
+                    atomicExch(g.error_flag, 3);
+                }
                 break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const uint32_t a_src = tiles + s * cfg::STAGE_BYTES;
-            const uint32_t b_src = a_src + cfg::A_BYTES;
-#pragma unroll
-            for (int k = 0; k < BK / 16; ++k) {
-                const uint64_t da = umma_desc(a_src + k * 32);
-                const uint64_t db = umma_desc(b_src + k * 32);
-                umma_f16(tmem_base, da, db, idesc, (kb | k) != 0 ? 1u : 0u);
-            }
-            umma_commit(empty0 + 8 * s);  // frees the stage once these MMAs have read it
-        }
-        umma_commit(accum_bar);  // accumulator complete (also arrives on the abort path)
-    }
-    __syncwarp();
+            const int row = m0 + quarter * 32 + lane;
+            const uint32_t tbase = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
 
-    // ---- epilogue: all four warps; warp w owns TMEM lanes 32w..32w+31 = tile rows 32w..32w+31
-    const bool ready = mbar_wait(accum_bar, 0);
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (!ready && lane == 0) atomicExch(error_flag, 3);
-    const bool good = ready && (*abort_flag == 0);
-    const int row = m0 + warp * 32 + lane;
-    if (good) {
-#pragma unroll 1
-        for (int c0 = 0; c0 < BN; c0 += 32) {
-            uint32_t r[32];
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c0;
-            asm volatile(
-                "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-                "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-                  "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
-                  "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
-                  "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
-                  "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-                : "r"(taddr)
-                : "memory");
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            if (row < M) {
-                float4* dst = reinterpret_cast<float4*>(C + (size_t)row * N + n0 + c0);
-#pragma unroll
-                for (int v = 0; v < 8; ++v) {
-                    float4 o = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
-                                           __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
-                    if (accumulate) {
-                        const float4 old = dst[v];
-                        o.x += old.x; o.y += old.y; o.z += old.z; o.w += old.w;
-                    }
-                    dst[v] = o;
+            RowDst rd;
+            rd.valid = row < M;
+            rd.s = 0;
+            rd.kvoff = 0;
+            if (EPI == EPI_QKV && rd.valid) {
+                const State& st = g.st;
+                const int i = row % st.W;
+                const int slot = (row / st.W) % g.S;
+                const int br = row / (st.W * g.S);
+                rd.valid = i < st.slot_n[slot];
+                if (rd.valid) {
+                    rd.s = st.slot_c[slot] + i;
+                    rd.kvoff = g.kv.offset(g.layer, br * st.Bmax + st.slot_img[slot], rd.s);
                 }
             }
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tbase + (uint32_t)c0, r);
+                const int col = n0 + c0;
+                if (EPI == EPI_STORE || EPI == EPI_ADD) {
+                    // registers -> swizzled staging tile (32 rows x 128 bytes) -> one TMA store / reduce-add
+                    // of the 32 x 32 block; rows past M are clipped by the tensor map
+                    const uint32_t sbuf = staging + (uint32_t)((warp - 2) * 2 + (int)(nchunk++ & 1u)) * 4096u;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const uint32_t addr = sbuf + (uint32_t)lane * 128u + (uint32_t)((v ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r[4 * v]),
+                                     "r"(r[4 * v + 1]), "r"(r[4 * v + 2]), "r"(r[4 * v + 3])
+                                     : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0 && m0 + quarter * 32 < M) {
+                        if (EPI == EPI_ADD)
+                            asm volatile(
+                                "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group "
+                                "[%0, {%1, %2}], [%3];" ::"l"(&map_c),
+                                "r"(col), "r"(m0 + quarter * 32), "r"(sbuf)
+                                : "memory");
+                        else
+                            asm volatile(
+                                "cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                                    &map_c),
+                                "r"(col), "r"(m0 + quarter * 32), "r"(sbuf)
+                                : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    continue;
+                }
+                if (!rd.valid) continue;
+                if (EPI == EPI_SWIGLU) {
+                    // columns (2f, 2f+1) = (gate_f, up_f)
+                    uint4* dst = reinterpret_cast<uint4*>(g.out + (size_t)row * (N / 2) + col / 2);
+                    uint32_t o[8];
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const float g0 = __uint_as_float(r[4 * v]), u0 = __uint_as_float(r[4 * v + 1]);
+                        const float g1 = __uint_as_float(r[4 * v + 2]), u1 = __uint_as_float(r[4 * v + 3]);
+                        o[v] = pack_bf16x2(g0 / (1.0f + expf(-g0)) * u0, g1 / (1.0f + expf(-g1)) * u1);
+                    }
+                    dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                    dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+                } else {  // EPI_QKV
+                    const State& st = g.st;
+                    const int D = st.D;
+                    const int sec = col / D, cs = col % D;  // 0 q, 1 k, 2 v; a tile never straddles sections
+                    uint32_t o[16];
+                    if (sec < 2) {
+                        const int half = st.dh / 2;
+                        const int e0 = (cs % st.dh) / 2;  // first rotation pair of this chunk within its head
+                        const float4* tab =
+                            reinterpret_cast<const float4*>(g.rope_cs + ((size_t)rd.s * half + e0) * 2);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            const float4 t = tab[v];  // cos, sin of pairs 2v and 2v+1
+                            const float a0 = __uint_as_float(r[4 * v]), b0 = __uint_as_float(r[4 * v + 1]);
+                            const float a1 = __uint_as_float(r[4 * v + 2]), b1 = __uint_as_float(r[4 * v + 3]);
+                            o[2 * v] = pack_bf16x2(a0 * t.x - b0 * t.y, a0 * t.y + b0 * t.x);
+                            o[2 * v + 1] = pack_bf16x2(a1 * t.z - b1 * t.w, a1 * t.w + b1 * t.z);
+                        }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 16; ++v)
+                            o[v] = pack_bf16x2(__uint_as_float(r[2 * v]), __uint_as_float(r[2 * v + 1]));
+                    }
+                    bf16* base = sec == 0 ? g.out + (size_t)row * D + cs
+                                          : (bf16*)(sec == 1 ? g.kv.k : g.kv.v) + rd.kvoff + cs;
+                    uint4* dst = reinterpret_cast<uint4*>(base);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) dst[v] = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+                }
+            }
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce0 + 8 * buf);
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
+    __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
@@ -258,66 +413,159 @@ bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows)
     const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN>
-cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, float* C, int M, int N, int K, int accumulate,
-                   int32_t* error_flag, cudaStream_t s) {
+int num_sms() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+// fp32 row-major [rows, N] output, box = 32 columns (128 bytes) x 32 rows, 128-byte swizzle.
+bool make_map_c(CUtensorMap* map, const float* base, int rows, int N) {
+    EncodeFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)N * 4};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int EPI>
+cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
+                   cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              Cfg<BN>::SMEM);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dim3 grid(N / BN, (M + BM - 1) / BM);
-    k_gemm_tcgen05<BN><<<grid, 128, Cfg<BN>::SMEM, s>>>(ma, mw, C, M, N, K, accumulate, error_flag);
+    const int tiles = (g.N / BN) * ((g.M + BM - 1) / BM);
+    const int grid = tiles < num_sms() ? tiles : num_sms();
+    k_gemm_tcgen05<BN, EPI><<<grid, NUM_THREADS, Cfg<BN>::SMEM, s>>>(ma, mw, mc, g);
     return cudaGetLastError();
 }
 
-}  // namespace
-
-int gemm_tcgen05_tile_n(int M, int N) {
-    const long tiles_m = (M + BM - 1) / BM;
-    if (N % 128 == 0 && tiles_m * (N / 128) >= 2 * 148) return 128;
-    if (N % 64 == 0 && tiles_m * (N / 64) >= 148) return 64;
-    if (N % 32 == 0) return 32;
-    return 64;
+template <int EPI>
+cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
+                      cudaStream_t s) {
+    switch (bn) {
+        case 32: return launch<32, EPI>(ma, mw, mc, g, s);
+        case 64: return launch<64, EPI>(ma, mw, mc, g, s);
+        case 128: return launch<128, EPI>(ma, mw, mc, g, s);
+        default: return launch<256, EPI>(ma, mw, mc, g, s);
+    }
 }
 
-int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
-                     int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int max_bn, cudaStream_t s, char* err,
+        size_t errlen) {
+    const int M = g.M, N = g.N, K = g.K;
     if (M <= 0) return 0;
-    if (K % BK != 0 || N % 32 != 0 || (((uintptr_t)A | (uintptr_t)W | (uintptr_t)C) & 15)) {
+    if (K % BK != 0 || N % 32 != 0 || (((uintptr_t)A | (uintptr_t)W) & 15)) {
         snprintf(err, errlen, "gemm: needs K %% 64 == 0, N %% 32 == 0 and 16-byte aligned operands (M=%d N=%d K=%d)",
                  M, N, K);
         return -1;
     }
-    const int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N);
-    if (N % bn != 0) {
+    static const int env_bn = getenv("HBSJD_GEMM_BN") ? atoi(getenv("HBSJD_GEMM_BN")) : 0;  // tuning aid
+    if (!force_bn && env_bn && N % env_bn == 0) force_bn = env_bn;
+    int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N);
+    while (bn > max_bn) bn >>= 1;
+    if (bn < 32 || N % bn != 0) {
         snprintf(err, errlen, "gemm: N=%d is not a multiple of the tile width %d", N, bn);
         return -1;
     }
-    CUtensorMap ma, mw;
+    CUtensorMap ma, mw, mc;
+    memset(&mc, 0, sizeof(mc));
+    if ((epi == EPI_STORE || epi == EPI_ADD) && !make_map_c(&mc, g.C, M, N)) {
+        snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed for the output (M=%d N=%d)", M, N);
+        return -3;
+    }
     if (!make_map(&ma, A, M, K, BM) || !make_map(&mw, W, N, K, bn)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
         return -3;
     }
     cudaError_t e;
-    switch (bn) {
-        case 32: e = launch<32>(ma, mw, C, M, N, K, accumulate, error_flag, s); break;
-        case 64: e = launch<64>(ma, mw, C, M, N, K, accumulate, error_flag, s); break;
-        case 128: e = launch<128>(ma, mw, C, M, N, K, accumulate, error_flag, s); break;
-        case 256: e = launch<256>(ma, mw, C, M, N, K, accumulate, error_flag, s); break;
-        default: snprintf(err, errlen, "gemm: unsupported tile width %d", bn); return -1;
+    switch (epi) {
+        case EPI_STORE: e = launch_bn<EPI_STORE>(bn, ma, mw, mc, g, s); break;
+        case EPI_ADD: e = launch_bn<EPI_ADD>(bn, ma, mw, mc, g, s); break;
+        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(bn, ma, mw, mc, g, s); break;
+        default: e = launch_bn<EPI_QKV>(bn, ma, mw, mc, g, s); break;
     }
     if (e != cudaSuccess) {
         snprintf(err, errlen, "gemm launch: %s", cudaGetErrorString(e));
         return -3;
     }
     return 0;
+}
+
+}  // namespace
+
+// Widest tile that still gives every SM a tile; small problems take narrower tiles.
+int gemm_tcgen05_tile_n(int M, int N) {
+    const long tiles_m = (M + BM - 1) / BM;
+    const int sms = 148;
+    for (int bn = 256; bn >= 64; bn >>= 1)
+        if (N % bn == 0 && tiles_m * (N / bn) >= sms) return bn;
+    for (int bn = 32; bn <= 256; bn <<= 1)
+        if (N % bn == 0) return bn;
+    return 32;
+}
+
+int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
+                     int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+    if ((uintptr_t)C & 15) {
+        snprintf(err, errlen, "gemm: C must be 16-byte aligned");
+        return -1;
+    }
+    GemmArgs g{};
+    g.C = C;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.error_flag = error_flag;
+    return run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, s, err, errlen);
+}
+
+int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K,
+                        int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+    GemmArgs g{};
+    g.out = act;
+    g.M = M;
+    g.N = F2;
+    g.K = K;
+    g.error_flag = error_flag;
+    return run(EPI_SWIGLU, A, W13_interleaved, g, 0, 256, s, err, errlen);
+}
+
+int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, int S, int layer,
+                     const float* rope_cs, const KvView& kv, int32_t* error_flag, cudaStream_t s, char* err,
+                     size_t errlen) {
+    GemmArgs g{};
+    g.out = q;
+    g.M = st.nb * S * st.W;
+    g.N = 3 * st.D;
+    g.K = st.D;
+    g.error_flag = error_flag;
+    g.st = st;
+    g.S = S;
+    g.layer = layer;
+    g.rope_cs = rope_cs;
+    g.kv = kv;
+    // a tile must lie inside one of the q / k / v sections and start on a rotation-pair boundary
+    int max_bn = 256;
+    while (st.D % max_bn != 0) max_bn >>= 1;
+    return run(EPI_QKV, A, Wqkv, g, 0, max_bn, s, err, errlen);
 }
 
 }  // namespace hbsjd
