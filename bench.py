@@ -234,7 +234,7 @@ def main():
         roof.update(bound="alu", peak=72.0, peak_source="fp32 CUDA-core FMA: 148 SMs x 128 lanes x 2 x 1.9 GHz")
         roof["frac"] = gemm_tflops / 72.0
     other = {}
-    for name in ("attention", "accept"):
+    for name in ("attention", "accept", "other"):
         c = prof[name]
         gbs = c["work"] / (c["ms"] * 1e-3) / 1e9 if c["ms"] > 0 else 0.0
         other[name] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",

@@ -162,6 +162,13 @@ int hbsjd_debug_read(hbsjd_ctx *c, int what, int index, void *host_dst, size_t m
  * M may be any size; bf16 needs N % 64 == 0 and K % 64 == 0; A, W 16-byte aligned. */
 int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate);
 
+/* Probability pipeline of the verification step on caller-supplied logits (Sec. 4.2: "verification uses the
+ * fused guided logits"): p = softmax(top_k((l_u + s (l_c - l_u)) / temperature)), ties at the k-th value kept.
+ * logits_c, logits_u: DEVICE fp32 [rows, V] (logits_u may be NULL: no guidance); probs: DEVICE fp32 [rows, V].
+ * V is the context's vocabulary.  Runs on the context's stream and waits for completion. */
+int hbsjd_probs(hbsjd_ctx *c, const float *logits_c, const float *logits_u, int rows, float cfg_scale,
+                float temperature, int top_k, float *probs);
+
 /* Per-kernel-class timing with CUDA events on the context's stream (off by default).  While enabled,
  * every launch of a timed class is bracketed by an event pair; totals accumulate until the next
  * hbsjd_profile(c, 1), which also resets them.  work = algorithmic FLOPs (GEMM: 2 M N K per launch) or

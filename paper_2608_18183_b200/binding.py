@@ -16,7 +16,7 @@ VERIFY_PROB, VERIFY_GREEDY = 0, 1
 EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
-EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
+EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
            "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_strerror", "hbsjd_last_error"]
 
 
@@ -73,6 +73,7 @@ def load():
                                          C.POINTER(hbsjd_stats)]
         L.hbsjd_profile.argtypes = [vp, C.c_int]
         L.hbsjd_profile_read.argtypes = [vp, C.POINTER(hbsjd_kernel_profile)]
+        L.hbsjd_probs.argtypes = [vp, vp, vp, C.c_int, C.c_float, C.c_float, C.c_int, vp]
         L.hbsjd_round.argtypes = [vp, C.POINTER(C.c_int)]
         L.hbsjd_tokens.argtypes = [vp, vp]
         L.hbsjd_destroy.argtypes = [vp]
@@ -164,6 +165,14 @@ class Context:
         self._check(self.lib.hbsjd_profile_read(self.h, C.byref(p)), "hbsjd_profile_read")
         return {n: dict(ms=p.ms[i], work=p.work[i], launches=p.launches[i]) for i, n in enumerate(PROF_CLASSES)} | {
             "dropped": p.dropped}
+
+    def hbsjd_probs(self, logits_c, logits_u=None, cfg_scale=1.0, temperature=1.0, top_k=0):
+        """Device fp32 [rows, V] logits -> device fp32 [rows, V] probabilities."""
+        out = self._torch.empty_like(logits_c)
+        self._check(self.lib.hbsjd_probs(self.h, logits_c.data_ptr(), None if logits_u is None else logits_u.data_ptr(),
+                                         logits_c.shape[0], cfg_scale, temperature, top_k, out.data_ptr()),
+                    "hbsjd_probs")
+        return out
 
     def hbsjd_round(self) -> int:
         live = C.c_int(0)

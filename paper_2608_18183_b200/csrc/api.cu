@@ -162,10 +162,16 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
     const KvView kv = kv_view(c);
     launch_embed<TA>(st, S, (const TA*)c->tok_emb, (const TA*)c->cls_emb, c->h, s);
     c->launches++;
+    // RMSNorm of the fp32 residual stream into the GEMM operand; algorithmic bytes: read fp32, write TA
+    auto norm = [&](const float* x, const void* gain) {
+        const int ps = prof_begin(c, HBSJD_PROF_OTHER, (double)M * D * (4.0 + sizeof(TA)));
+        launch_rmsnorm<TA>(x, (const TA*)gain, (TA*)c->a, M, D, c->d.rms_eps, s);
+        prof_end(c, ps);
+    };
     for (int l = 0; l < st.L; ++l) {
         const LayerW& w = c->layers[l];
         int rc;
-        launch_rmsnorm<TA>(c->h, (const TA*)w.g_attn, (TA*)c->a, M, D, c->d.rms_eps, s);
+        norm(c->h, w.g_attn);
         if constexpr (std::is_same<TA, bf16>::value) {
             // QKV projection with RoPE and the paged KV write in its epilogue
             const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D);
@@ -193,7 +199,7 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
             c->launches++;
         }
         if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1))) return rc;
-        launch_rmsnorm<TA>(c->h, (const TA*)w.g_ffn, (TA*)c->a, M, D, c->d.rms_eps, s);
+        norm(c->h, w.g_ffn);
         c->launches++;
         if constexpr (std::is_same<TA, bf16>::value) {
             // gate/up projection with SwiGLU in its epilogue (gate and up rows interleaved at load time)
@@ -211,7 +217,7 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
         if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1))) return rc;
     }
     if (want_logits) {
-        launch_rmsnorm<TA>(c->h, (const TA*)c->g_out, (TA*)c->a, M, D, c->d.rms_eps, s);
+        norm(c->h, c->g_out);
         c->launches++;
         int rc;
         if ((rc = gemm<TA>(c, c->a, c->w_head, c->logits, M, st.V, D, 0))) return rc;
@@ -657,6 +663,17 @@ int hbsjd_rollout_host(hbsjd_ctx* c, int batch, const int32_t* prefix_tokens, co
     const int rc = hbsjd_rollout(c, batch, c->stage_tok, c->stage_len, c->stage_lab, p, c->stage_out, stats);
     if (rc) return rc;
     CK(cudaMemcpyAsync(out_tokens, c->stage_out, bt, cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
+}
+
+int hbsjd_probs(hbsjd_ctx* c, const float* logits_c, const float* logits_u, int rows, float cfg_scale,
+                float temperature, int top_k, float* probs) {
+    if (!c || !logits_c || !probs || rows < 1 || !(temperature > 0.f) || top_k < 0 ||
+        (((uintptr_t)logits_c | (uintptr_t)logits_u | (uintptr_t)probs) & 15))
+        return HBSJD_EINVAL;
+    launch_probs(logits_c, logits_u, rows, c->d.vocab, cfg_scale, temperature, top_k, probs, c->stream);
+    CK(cudaGetLastError());
     CK(cudaStreamSynchronize(c->stream));
     return HBSJD_OK;
 }

@@ -57,6 +57,8 @@ template <int QB, int HPC>
 __global__ void __launch_bounds__(QB * HPC * 32) k_attention_mma(State st, int S, int layer,
                                                                  const bf16* __restrict__ q, KvView kv,
                                                                  bf16* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int NT = QB * HPC * 32;
     constexpr int HEAD_STAGE = 2 * KB * DH * 2;       // K + V bytes of one head in one stage (8 KB)
     constexpr int STAGE_BYTES = HPC * HEAD_STAGE;
@@ -234,7 +236,7 @@ void launch_cfg(const State& st, int S, int layer, const bf16* q, KvView kv, bf1
         configured = true;
     }
     dim3 grid(st.nb * S, st.Hh / HPC);
-    k_attention_mma<QB, HPC><<<grid, QB * HPC * 32, smem, s>>>(st, S, layer, q, kv, out);
+    launch_k(k_attention_mma<QB, HPC>, dim3(grid), dim3(QB * HPC * 32), smem, s, st, S, layer, q, kv, out);
 }
 
 template <int HPC>

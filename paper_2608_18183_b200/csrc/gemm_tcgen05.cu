@@ -162,6 +162,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                                                               const GemmArgs g) {
     using cfg = Cfg<BN>;
     extern __shared__ unsigned char smem_raw[];
+    pdl_trigger();
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // 1024-byte aligned tile ring
     const uint32_t staging = tiles + cfg::STAGES * cfg::STAGE_BYTES;  // 1024-byte aligned
@@ -202,6 +203,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();  // everything above is on-chip set-up; operands of the previous kernel are read from here on
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -453,8 +455,7 @@ cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorM
     }
     const int tiles = (g.N / BN) * ((g.M + BM - 1) / BM);
     const int grid = tiles < num_sms() ? tiles : num_sms();
-    k_gemm_tcgen05<BN, EPI><<<grid, NUM_THREADS, Cfg<BN>::SMEM, s>>>(ma, mw, mc, g);
-    return cudaGetLastError();
+    return launch_k(k_gemm_tcgen05<BN, EPI>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<BN>::SMEM, s, ma, mw, mc, g);
 }
 
 template <int EPI>

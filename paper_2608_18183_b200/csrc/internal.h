@@ -77,6 +77,8 @@ void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s);
 void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s);
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s);
 int accept_smem_bytes(int V);
+void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
+                  float* p, cudaStream_t s);
 
 // ---- tcgen05 GEMM (gemm_tcgen05.cu)
 // C[M,N] fp32 (+)= A[M,K] bf16 . W[N,K]^T bf16.  force_bn: 0 = choose the tile width from the shape.

@@ -8,6 +8,8 @@ namespace hbsjd {
 // One block.  Builds the slot tables of the next forward.  Full: slot b = image b, n = 0 for inactive
 // images.  Compact: active images gathered in increasing image order (block-wide exclusive scan).
 __global__ void k_setup(State st, int phase, int compact) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ int warp_tot[32];
     __shared__ int carry, sum_keys, sum_n;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
@@ -69,13 +71,15 @@ __global__ void k_setup(State st, int phase, int compact) {
 }
 
 void launch_setup(const State& st, int phase, int compact, cudaStream_t s) {
-    k_setup<<<1, 1024, 0, s>>>(st, phase, compact);
+    launch_k(k_setup, dim3(1), dim3(1024), 0, s, st, phase, compact);
 }
 
 // ------------------------------------------------------------------ embedding gather
 template <typename TA>
 __global__ void k_embed(State st, int S, const TA* __restrict__ tok_emb, const TA* __restrict__ cls_emb,
                         float* __restrict__ h) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x;
     const int i = row % st.W;
     const int slot = (row / st.W) % S;
@@ -100,15 +104,61 @@ __global__ void k_embed(State st, int S, const TA* __restrict__ tok_emb, const T
 
 template <typename TA>
 void launch_embed(const State& st, int S, const TA* tok_emb, const TA* cls_emb, float* h, cudaStream_t s) {
-    k_embed<TA><<<st.nb * S * st.W, 128, 0, s>>>(st, S, tok_emb, cls_emb, h);
+    launch_k(k_embed<TA>, dim3(st.nb * S * st.W), dim3(128), 0, s, st, S, tok_emb, cls_emb, h);
 }
 template void launch_embed<float>(const State&, int, const float*, const float*, float*, cudaStream_t);
 template void launch_embed<bf16>(const State&, int, const bf16*, const bf16*, float*, cudaStream_t);
 
 // ------------------------------------------------------------------ RMSNorm: out = x * rsqrt(mean(x^2)+eps) * g
+// One warp per row; the row stays in registers between the two passes (D <= 2048 through the vector path).
+// The sum of squares is reduced in a fixed order that depends on D only.
+template <typename TA, int VEC_ITERS>
+__global__ void __launch_bounds__(256) k_rmsnorm_warp(const float* __restrict__ h, const TA* __restrict__ gain,
+                                                      TA* __restrict__ out, int M, int D, float eps) {
+    pdl_trigger();
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= M) return;
+    const float4* x4 = reinterpret_cast<const float4*>(h + (size_t)row * D);
+    float4 v[VEC_ITERS];
+    float ss = 0.f;
+#pragma unroll
+    for (int it = 0; it < VEC_ITERS; ++it) {
+        const int idx = it * 32 + lane;
+        if (idx * 4 < D) {
+            v[it] = x4[idx];
+            ss += v[it].x * v[it].x + v[it].y * v[it].y + v[it].z * v[it].z + v[it].w * v[it].w;
+        }
+    }
+    ss = warp_sum(ss);
+    const float r = 1.0f / sqrtf(ss / (float)D + eps);
+    TA* o = out + (size_t)row * D;
+#pragma unroll
+    for (int it = 0; it < VEC_ITERS; ++it) {
+        const int idx = it * 32 + lane;
+        if (idx * 4 < D) {
+            const int e = idx * 4;
+            const float a = v[it].x * r * to_f<TA>(gain[e]), b = v[it].y * r * to_f<TA>(gain[e + 1]);
+            const float c = v[it].z * r * to_f<TA>(gain[e + 2]), d = v[it].w * r * to_f<TA>(gain[e + 3]);
+            if constexpr (sizeof(TA) == 2) {
+                __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(o + e) = pk;
+            } else {
+                *reinterpret_cast<float4*>(o + e) = make_float4(a, b, c, d);
+            }
+        }
+    }
+}
+
 template <typename TA>
 __global__ void k_rmsnorm(const float* __restrict__ h, const TA* __restrict__ gain, TA* __restrict__ out, int D,
                           float eps) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float red[32];
     const int row = blockIdx.x;
     const float* x = h + (size_t)row * D;
@@ -126,7 +176,14 @@ __global__ void k_rmsnorm(const float* __restrict__ h, const TA* __restrict__ ga
 
 template <typename TA>
 void launch_rmsnorm(const float* h, const TA* gain, TA* out, int M, int D, float eps, cudaStream_t s) {
-    k_rmsnorm<TA><<<M, 128, 0, s>>>(h, gain, out, D, eps);
+    if (D % 4 == 0 && D <= 2048) {
+        const int grid = (M + 7) / 8;
+        if (D <= 512) launch_k(k_rmsnorm_warp<TA, 4>, dim3(grid), dim3(256), 0, s, h, gain, out, M, D, eps);
+        else if (D <= 1024) launch_k(k_rmsnorm_warp<TA, 8>, dim3(grid), dim3(256), 0, s, h, gain, out, M, D, eps);
+        else launch_k(k_rmsnorm_warp<TA, 16>, dim3(grid), dim3(256), 0, s, h, gain, out, M, D, eps);
+    } else {
+        launch_k(k_rmsnorm<TA>, dim3(M), dim3(128), 0, s, h, gain, out, D, eps);
+    }
 }
 template void launch_rmsnorm<float>(const float*, const float*, float*, int, int, float, cudaStream_t);
 template void launch_rmsnorm<bf16>(const float*, const bf16*, bf16*, int, int, float, cudaStream_t);
@@ -136,6 +193,8 @@ template void launch_rmsnorm<bf16>(const float*, const bf16*, bf16*, int, int, f
 template <typename TA>
 __global__ void k_rope_kv(State st, int S, int layer, const float* __restrict__ qkv,
                           const float* __restrict__ rope_cs, TA* __restrict__ q, KvView kv) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.x;
     const int i = row % st.W;
     const int slot = (row / st.W) % S;
@@ -174,7 +233,7 @@ __global__ void k_rope_kv(State st, int S, int layer, const float* __restrict__ 
 template <typename TA>
 void launch_rope_kv(const State& st, int S, int layer, const float* qkv, const float* rope_cs, TA* q, KvView kv,
                     cudaStream_t s) {
-    k_rope_kv<TA><<<st.nb * S * st.W, 128, 0, s>>>(st, S, layer, qkv, rope_cs, q, kv);
+    launch_k(k_rope_kv<TA>, dim3(st.nb * S * st.W), dim3(128), 0, s, st, S, layer, qkv, rope_cs, q, kv);
 }
 template void launch_rope_kv<float>(const State&, int, int, const float*, const float*, float*, KvView, cudaStream_t);
 template void launch_rope_kv<bf16>(const State&, int, int, const float*, const float*, bf16*, KvView, cudaStream_t);
@@ -185,6 +244,8 @@ template void launch_rope_kv<bf16>(const State&, int, int, const float*, const f
 template <typename TA>
 __global__ void k_attention_ref(State st, int S, int layer, const TA* __restrict__ q, KvView kv,
                                 TA* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ float smem[];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     const int row = blockIdx.x;
@@ -242,7 +303,7 @@ void launch_attention_ref(const State& st, int S, int layer, const TA* q, KvView
     const int nw = 4;
     dim3 grid(st.nb * S * st.W, (st.Hh + nw - 1) / nw);
     const size_t smem = (size_t)nw * (st.T + st.dh) * sizeof(float);
-    k_attention_ref<TA><<<grid, nw * 32, smem, s>>>(st, S, layer, q, kv, out);
+    launch_k(k_attention_ref<TA>, dim3(grid), dim3(nw * 32), smem, s, st, S, layer, q, kv, out);
 }
 template void launch_attention_ref<float>(const State&, int, int, const float*, KvView, float*, cudaStream_t);
 template void launch_attention_ref<bf16>(const State&, int, int, const bf16*, KvView, bf16*, cudaStream_t);
@@ -250,6 +311,8 @@ template void launch_attention_ref<bf16>(const State&, int, int, const bf16*, Kv
 // ------------------------------------------------------------------ SwiGLU: act = silu(gate) * up
 template <typename TA>
 __global__ void k_swiglu(const float* __restrict__ gu, TA* __restrict__ act, int F) {
+    pdl_trigger();
+    pdl_wait();
     const int row = blockIdx.y;
     const int f = blockIdx.x * blockDim.x + threadIdx.x;
     if (f >= F) return;
@@ -260,7 +323,7 @@ __global__ void k_swiglu(const float* __restrict__ gu, TA* __restrict__ act, int
 template <typename TA>
 void launch_swiglu(const float* gu, TA* act, int M, int F, cudaStream_t s) {
     dim3 grid((F + 255) / 256, M);
-    k_swiglu<TA><<<grid, 256, 0, s>>>(gu, act, F);
+    launch_k(k_swiglu<TA>, dim3(grid), dim3(256), 0, s, gu, act, F);
 }
 template void launch_swiglu<float>(const float*, float*, int, int, cudaStream_t);
 template void launch_swiglu<bf16>(const float*, bf16*, int, int, cudaStream_t);
@@ -270,6 +333,8 @@ template void launch_swiglu<bf16>(const float*, bf16*, int, int, cudaStream_t);
 template <typename TA>
 __global__ void __launch_bounds__(256) k_gemm_simt(const TA* __restrict__ A, const TA* __restrict__ W,
                                                    float* __restrict__ C, int M, int N, int K, int accumulate) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float As[16][64 + 4];
     __shared__ float Bs[16][64 + 4];
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
@@ -319,7 +384,7 @@ __global__ void __launch_bounds__(256) k_gemm_simt(const TA* __restrict__ A, con
 template <typename TA>
 void launch_gemm_simt(const TA* A, const TA* W, float* C, int M, int N, int K, int accumulate, cudaStream_t s) {
     dim3 grid((N + 63) / 64, (M + 63) / 64);
-    k_gemm_simt<TA><<<grid, 256, 0, s>>>(A, W, C, M, N, K, accumulate);
+    launch_k(k_gemm_simt<TA>, dim3(grid), dim3(256), 0, s, A, W, C, M, N, K, accumulate);
 }
 template void launch_gemm_simt<float>(const float*, const float*, float*, int, int, int, int, cudaStream_t);
 template void launch_gemm_simt<bf16>(const bf16*, const bf16*, float*, int, int, int, int, cudaStream_t);

@@ -7,6 +7,8 @@ namespace hbsjd {
 // ------------------------------------------------------------------ state init (Sec. 4.2 "Independent rollout states")
 __global__ void k_init_state(State st, const int32_t* __restrict__ prefix_tokens,
                              const int32_t* __restrict__ prefix_len, const int32_t* __restrict__ labels) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x;
     const int k = prefix_len[b];
     int32_t* seq = st.seq + (size_t)b * (st.T + 1);
@@ -31,10 +33,12 @@ __global__ void k_init_state(State st, const int32_t* __restrict__ prefix_tokens
 
 void launch_init_state(const State& st, const int32_t* prefix_tokens, const int32_t* prefix_len,
                        const int32_t* labels, cudaStream_t s) {
-    k_init_state<<<st.B, 128, 0, s>>>(st, prefix_tokens, prefix_len, labels);
+    launch_k(k_init_state, dim3(st.B), dim3(128), 0, s, st, prefix_tokens, prefix_len, labels);
 }
 
 __global__ void k_prefill_advance(State st, int S) {
+    pdl_trigger();
+    pdl_wait();
     const int slot = blockIdx.x * blockDim.x + threadIdx.x;
     if (slot >= S) return;
     const int n = st.slot_n[slot];
@@ -42,12 +46,14 @@ __global__ void k_prefill_advance(State st, int S) {
 }
 
 void launch_prefill_advance(const State& st, int S, cudaStream_t s) {
-    k_prefill_advance<<<(S + 127) / 128, 128, 0, s>>>(st, S);
+    launch_k(k_prefill_advance, dim3((S + 127) / 128), dim3(128), 0, s, st, S);
 }
 
 // Initial window: every draft is the token H positions back, or a keyed uniform token where that
 // position does not exist; all are point-mass proposals.  Reserved round value 0xFFFFFFFF.
 __global__ void k_init_window(State st, uint32_t seed_lo, uint32_t seed_hi) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= st.B) return;
     const int c = st.cursor[b];
@@ -69,17 +75,19 @@ __global__ void k_init_window(State st, uint32_t seed_lo, uint32_t seed_hi) {
 }
 
 void launch_init_window(const State& st, uint32_t seed_lo, uint32_t seed_hi, cudaStream_t s) {
-    k_init_window<<<(st.B + 63) / 64, 64, 0, s>>>(st, seed_lo, seed_hi);
+    launch_k(k_init_window, dim3((st.B + 63) / 64), dim3(64), 0, s, st, seed_lo, seed_hi);
 }
 
 __global__ void k_export_tokens(State st, int32_t* __restrict__ out) {
+    pdl_trigger();
+    pdl_wait();
     const int b = blockIdx.x;
     for (int t = threadIdx.x; t < st.T; t += blockDim.x)
         out[(size_t)b * st.T + t] = st.seq[(size_t)b * (st.T + 1) + t + 1];
 }
 
 void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s) {
-    k_export_tokens<<<st.B, 128, 0, s>>>(st, out);
+    launch_k(k_export_tokens, dim3(st.B), dim3(128), 0, s, st, out);
 }
 
 // ------------------------------------------------------------------ probability pipeline + verification
@@ -180,7 +188,214 @@ __device__ int block_sample(const float* a, int V, uint32_t word, AccShared& sh)
     return sh.result;
 }
 
+// Key of the k-th largest of g[0..V) by radix select, one byte per pass from the top (exact for any input).
+__device__ unsigned int radix_select(const float* g, int V, unsigned int k, AccShared& sh) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    if (tid == 0) {
+        sh.sel_prefix = 0u;
+        sh.sel_k = k;
+    }
+    for (int pass = 0; pass < 4; ++pass) {
+        const int shift = 24 - 8 * pass;
+        const unsigned int mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
+        for (int x = lane; x < 256; x += 32) sh.hist[wid][x] = 0u;
+        __syncthreads();
+        const unsigned int prefix = sh.sel_prefix;
+        for (int v = tid; v < V; v += ACC_THREADS) {
+            const unsigned int key = float_key(g[v]);
+            if ((key & mask) == prefix) atomicAdd(&sh.hist[wid][(key >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (wid == 0) {
+            // lane owns 8 consecutive bins; scan from the top bin downwards
+            unsigned int cnt[8], tot = 0;
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                unsigned int s = 0;
+                for (int w = 0; w < ACC_WARPS; ++w) s += sh.hist[w][lane * 8 + x];
+                cnt[x] = s;
+                tot += s;
+            }
+            unsigned int incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int tt = __shfl_down_sync(0xffffffffu, incl, o);
+                if (lane + o < 32) incl += tt;
+            }
+            unsigned int above = incl - tot;
+            const unsigned int kk = sh.sel_k;
+            if (above < kk && kk <= above + tot) {  // exactly one lane
+#pragma unroll
+                for (int x = 7; x >= 0; --x) {
+                    if (above < kk && kk <= above + cnt[x]) {
+                        sh.sel_prefix = prefix | ((unsigned int)(lane * 8 + x) << shift);
+                        sh.sel_k = kk - above;
+                        above = 0xFFFFFFFFu;  // done
+                    } else if (above != 0xFFFFFFFFu) {
+                        above += cnt[x];
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    return sh.sel_prefix;
+}
+
+// Key of the k-th largest of g[0..V), 0 < k < V.  One pass builds a 1024-bin histogram over [min, max]
+// with a monotone binning (a higher bin holds strictly larger values), which locates the bin of the k-th
+// largest and its rank inside that bin; the few entries of that bin are then ranked exactly against one
+// another.  Falls back to the radix select when that bin is crowded.  *gmax receives max(g).
+constexpr int SEL_BINS = 1024;
+constexpr int SEL_CAP = 2048;
+__device__ unsigned int topk_threshold(const float* g, int V, unsigned int k, AccShared& sh, float* gmax) {
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    unsigned int* hist = &sh.hist[0][0];       // [SEL_BINS]
+    unsigned int* cand = hist + SEL_BINS;      // [SEL_CAP] keys of the entries of the selected bin
+    float mn = INFINITY, mx = -INFINITY;
+    for (int v = tid; v < V; v += ACC_THREADS) {
+        const float x = g[v];
+        mn = fminf(mn, x);
+        mx = fmaxf(mx, x);
+    }
+    mx = block_max(mx, sh);
+    mn = -block_max(-mn, sh);
+    *gmax = mx;
+    if (!(mx > mn)) return float_key(mn);  // all entries equal: everything is kept
+    const float scale = (float)SEL_BINS / (mx - mn);
+    for (int x = tid; x < SEL_BINS; x += ACC_THREADS) hist[x] = 0u;
+    if (tid == 0) {
+        sh.sel_prefix = 0u;  // selected bin
+        sh.sel_k = 0u;       // rank of the k-th largest inside it (1-based, from the top)
+        sh.result = 0;       // candidate count
+    }
+    __syncthreads();
+    for (int v = tid; v < V; v += ACC_THREADS) {
+        const int b = min(SEL_BINS - 1, (int)((g[v] - mn) * scale));
+        atomicAdd(&hist[b], 1u);
+    }
+    __syncthreads();
+    if (wid == 0) {
+        unsigned int tot = 0;
+        for (int x = 0; x < 32; ++x) tot += hist[lane * 32 + x];
+        unsigned int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned int tt = __shfl_down_sync(0xffffffffu, incl, o);
+            if (lane + o < 32) incl += tt;
+        }
+        unsigned int above = incl - tot;
+        if (above < k && k <= above + tot) {  // exactly one lane
+            for (int x = 31; x >= 0; --x) {
+                const unsigned int c = hist[lane * 32 + x];
+                if (k <= above + c) {
+                    sh.sel_prefix = (unsigned int)(lane * 32 + x);
+                    sh.sel_k = k - above;
+                    break;
+                }
+                above += c;
+            }
+        }
+    }
+    __syncthreads();
+    const int bsel = (int)sh.sel_prefix;
+    const unsigned int krem = sh.sel_k;
+    for (int v = tid; v < V; v += ACC_THREADS) {
+        const float x = g[v];
+        if (min(SEL_BINS - 1, (int)((x - mn) * scale)) == bsel) {
+            const int slot = atomicAdd(&sh.result, 1);
+            if (slot < SEL_CAP) cand[slot] = float_key(x);
+        }
+    }
+    __syncthreads();
+    const int nc = sh.result;
+    __syncthreads();
+    if (nc > SEL_CAP) return radix_select(g, V, k, sh);
+    // the value with (#strictly greater) < krem <= (#greater or equal) is the krem-th largest of the bin
+    for (int i = tid; i < nc; i += ACC_THREADS) {
+        const unsigned int ki = cand[i];
+        unsigned int gt = 0, ge = 0;
+        for (int j = 0; j < nc; ++j) {
+            const unsigned int kj = cand[j];
+            gt += kj > ki;
+            ge += kj >= ki;
+        }
+        if (gt < krem && krem <= ge) sh.sel_prefix = ki;  // every such thread writes the same key
+    }
+    __syncthreads();
+    const unsigned int theta = sh.sel_prefix;
+    __syncthreads();
+    return theta;
+}
+
+// Probability pipeline of one position, all threads of the CTA: guided = l_u + s (l_c - l_u); divided by
+// the temperature; top-k threshold (ties kept); softmax in fp32.  Leaves p in g[0..V) (shared memory) and
+// writes it to pout.  Ends with a block-wide barrier.
+__device__ void prob_pipeline(float* g, const float* __restrict__ lc, const float* __restrict__ lu, int V,
+                              float cfg_scale, float temperature, int top_k, float* __restrict__ pout,
+                              AccShared& sh) {
+    const int tid = threadIdx.x;
+    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+        float4 x = *reinterpret_cast<const float4*>(lc + v);
+        if (lu) {
+            const float4 y = *reinterpret_cast<const float4*>(lu + v);
+            x.x = __fadd_rn(y.x, __fmul_rn(cfg_scale, __fsub_rn(x.x, y.x)));
+            x.y = __fadd_rn(y.y, __fmul_rn(cfg_scale, __fsub_rn(x.y, y.y)));
+            x.z = __fadd_rn(y.z, __fmul_rn(cfg_scale, __fsub_rn(x.z, y.z)));
+            x.w = __fadd_rn(y.w, __fmul_rn(cfg_scale, __fsub_rn(x.w, y.w)));
+        }
+        x.x = __fdiv_rn(x.x, temperature);
+        x.y = __fdiv_rn(x.y, temperature);
+        x.z = __fdiv_rn(x.z, temperature);
+        x.w = __fdiv_rn(x.w, temperature);
+        *reinterpret_cast<float4*>(g + v) = x;
+    }
+    __syncthreads();
+    unsigned int theta = 0u;
+    float mx;
+    if (top_k > 0 && top_k < V) {
+        theta = topk_threshold(g, V, (unsigned int)top_k, sh, &mx);  // the largest entry is always kept
+    } else {
+        mx = -INFINITY;
+        for (int v = tid; v < V; v += ACC_THREADS) mx = fmaxf(mx, g[v]);
+        mx = block_max(mx, sh);
+    }
+    float part = 0.f;
+    for (int v = tid; v < V; v += ACC_THREADS) {
+        const float x = g[v];
+        const float e = float_key(x) >= theta ? expf(x - mx) : 0.f;
+        g[v] = e;
+        part += e;
+    }
+    const float den = block_sum(part, sh);
+    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+        float4 e = *reinterpret_cast<float4*>(g + v);
+        e.x = __fdiv_rn(e.x, den);
+        e.y = __fdiv_rn(e.y, den);
+        e.z = __fdiv_rn(e.z, den);
+        e.w = __fdiv_rn(e.w, den);
+        *reinterpret_cast<float4*>(g + v) = e;
+        *reinterpret_cast<float4*>(pout + v) = e;
+    }
+    __syncthreads();
+}
+
+// Stand-alone probability pipeline: one CTA per row of logits.
+__global__ void __launch_bounds__(ACC_THREADS) k_probs(const float* __restrict__ lc, const float* __restrict__ lu,
+                                                       int V, float cfg_scale, float temperature, int top_k,
+                                                       float* __restrict__ p) {
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* g = (float*)smem_raw;
+    AccShared& sh = *(AccShared*)(smem_raw + (size_t)V * sizeof(float));
+    const size_t row = blockIdx.x;
+    prob_pipeline(g, lc + row * V, lu ? lu + row * V : nullptr, V, cfg_scale, temperature, top_k, p + row * V, sh);
+}
+
 __global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArgs a) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     float* g = (float*)smem_raw;  // [V]
     AccShared& sh = *(AccShared*)(smem_raw + (size_t)st.V * sizeof(float));
@@ -195,106 +410,8 @@ __global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArg
     const float* lu = a.logits + ((size_t)(a.S + slot) * st.W + i) * V;
     if (tid == 0) philox4x32_10((uint32_t)img, (uint32_t)t, a.round, 0u, a.seed_lo, a.seed_hi, sh.words);
 
-    // guided logits / temperature
-    const bool cfg = st.nb == 2;
-    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
-        float4 x = *reinterpret_cast<const float4*>(lc + v);
-        if (cfg) {
-            const float4 y = *reinterpret_cast<const float4*>(lu + v);
-            x.x = __fadd_rn(y.x, __fmul_rn(a.cfg_scale, __fsub_rn(x.x, y.x)));
-            x.y = __fadd_rn(y.y, __fmul_rn(a.cfg_scale, __fsub_rn(x.y, y.y)));
-            x.z = __fadd_rn(y.z, __fmul_rn(a.cfg_scale, __fsub_rn(x.z, y.z)));
-            x.w = __fadd_rn(y.w, __fmul_rn(a.cfg_scale, __fsub_rn(x.w, y.w)));
-        }
-        x.x = __fdiv_rn(x.x, a.temperature);
-        x.y = __fdiv_rn(x.y, a.temperature);
-        x.z = __fdiv_rn(x.z, a.temperature);
-        x.w = __fdiv_rn(x.w, a.temperature);
-        *reinterpret_cast<float4*>(g + v) = x;
-    }
-    __syncthreads();
-
-    // top-k threshold: key of the k-th largest value, one byte per pass from the top
-    unsigned int theta = 0u;
-    if (a.top_k > 0 && a.top_k < V) {
-        if (tid == 0) {
-            sh.sel_prefix = 0u;
-            sh.sel_k = (unsigned int)a.top_k;
-        }
-        for (int pass = 0; pass < 4; ++pass) {
-            const int shift = 24 - 8 * pass;
-            const unsigned int mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-            for (int x = lane; x < 256; x += 32) sh.hist[wid][x] = 0u;
-            __syncthreads();
-            const unsigned int prefix = sh.sel_prefix;
-            for (int v = tid; v < V; v += ACC_THREADS) {
-                const unsigned int key = float_key(g[v]);
-                if ((key & mask) == prefix) atomicAdd(&sh.hist[wid][(key >> shift) & 255u], 1u);
-            }
-            __syncthreads();
-            if (wid == 0) {
-                // lane owns 8 consecutive bins (bins 8*lane .. 8*lane+7); scan from the top bin downwards
-                unsigned int cnt[8], tot = 0;
-#pragma unroll
-                for (int x = 0; x < 8; ++x) {
-                    unsigned int s = 0;
-                    for (int w = 0; w < ACC_WARPS; ++w) s += sh.hist[w][lane * 8 + x];
-                    cnt[x] = s;
-                    tot += s;
-                }
-                // suffix sum over lanes: above = elements in bins of higher lanes
-                unsigned int incl = tot;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const unsigned int tt = __shfl_down_sync(0xffffffffu, incl, o);
-                    if (lane + o < 32) incl += tt;
-                }
-                unsigned int above = incl - tot;
-                const unsigned int k = sh.sel_k;
-                if (above < k && k <= above + tot) {  // exactly one lane
-#pragma unroll
-                    for (int x = 7; x >= 0; --x) {
-                        if (above < k && k <= above + cnt[x]) {
-                            sh.sel_prefix = prefix | ((unsigned int)(lane * 8 + x) << shift);
-                            sh.sel_k = k - above;
-                            above = 0xFFFFFFFFu;  // done
-                        } else if (above != 0xFFFFFFFFu) {
-                            above += cnt[x];
-                        }
-                    }
-                }
-            }
-            __syncthreads();
-        }
-        theta = sh.sel_prefix;
-    }
-
-    // softmax over the kept entries
-    float mx = -INFINITY;
-    for (int v = tid; v < V; v += ACC_THREADS) {
-        const float x = g[v];
-        if (float_key(x) >= theta) mx = fmaxf(mx, x);
-    }
-    mx = block_max(mx, sh);
-    float part = 0.f;
-    for (int v = tid; v < V; v += ACC_THREADS) {
-        const float x = g[v];
-        const float e = float_key(x) >= theta ? expf(x - mx) : 0.f;
-        g[v] = e;
-        part += e;
-    }
-    const float den = block_sum(part, sh);
     float* pout = a.pcur + ((size_t)img * st.Wmax + i) * V;
-    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
-        float4 e = *reinterpret_cast<float4*>(g + v);
-        e.x = __fdiv_rn(e.x, den);
-        e.y = __fdiv_rn(e.y, den);
-        e.z = __fdiv_rn(e.z, den);
-        e.w = __fdiv_rn(e.w, den);
-        *reinterpret_cast<float4*>(g + v) = e;
-        *reinterpret_cast<float4*>(pout + v) = e;
-    }
-    __syncthreads();
+    prob_pipeline(g, lc, st.nb == 2 ? lu : nullptr, V, a.cfg_scale, a.temperature, a.top_k, pout, sh);
 
     const size_t oidx = (size_t)img * st.Wmax + i;
     const bool last = (i == n - 1);
@@ -385,6 +502,17 @@ __global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArg
 
 int accept_smem_bytes(int V) { return V * (int)sizeof(float) + (int)sizeof(AccShared); }
 
+void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
+                  float* p, cudaStream_t s) {
+    static int configured_bytes = 0;
+    const int bytes = accept_smem_bytes(V);
+    if (bytes > configured_bytes) {
+        cudaFuncSetAttribute(k_probs, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        configured_bytes = bytes;
+    }
+    launch_k(k_probs, dim3(rows), dim3(ACC_THREADS), bytes, s, lc, lu, V, cfg_scale, temperature, top_k, p);
+}
+
 void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
     static int configured_bytes = 0;
     const int bytes = accept_smem_bytes(st.V);
@@ -393,7 +521,7 @@ void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
         configured_bytes = bytes;
     }
     dim3 grid(st.W, a.S);
-    k_prob_accept<<<grid, ACC_THREADS, accept_smem_bytes(st.V), s>>>(st, a);
+    launch_k(k_prob_accept, dim3(grid), dim3(ACC_THREADS), accept_smem_bytes(st.V), s, st, a);
 }
 
 // ------------------------------------------------------------------ commit + refresh (one warp per slot)
@@ -401,6 +529,8 @@ void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
 // (or bonus) token, advances the cursor -- the KV commit is this cursor move: entries at and after the
 // new cursor are recomputed by the next forward (Sec. 4.2 "Independent progress") -- and rebuilds the window.
 __global__ void k_commit(State st, AcceptArgs a) {
+    pdl_trigger();
+    pdl_wait();
     const int lane = threadIdx.x & 31;
     const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (slot >= a.S) return;
@@ -454,7 +584,7 @@ __global__ void k_commit(State st, AcceptArgs a) {
 }
 
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s) {
-    k_commit<<<(a.S + 3) / 4, 128, 0, s>>>(st, a);
+    launch_k(k_commit, dim3((a.S + 3) / 4), dim3(128), 0, s, st, a);
 }
 
 }  // namespace hbsjd
