@@ -169,6 +169,28 @@ int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int 
 int hbsjd_probs(hbsjd_ctx *c, const float *logits_c, const float *logits_u, int rows, float cfg_scale,
                 float temperature, int top_k, float *probs);
 
+/* Verification step of one round on caller-supplied logits (Sec. 4.2, Eq. 5 / Eq. 4): probability pipeline,
+ * accept test of every draft left to right, residual resampling at the first reject (or the bonus token),
+ * commit, cursor advance and draft refresh, for `batch` images in Full layout.  All pointers DEVICE.
+ *   logits  fp32 [branches, batch, window, V]  branch 0 conditional, branch 1 unconditional (branches = 1 or 2)
+ *   q_prev  fp32 [batch, window, V]  previous round's probabilities (row t - qbase - 1 = proposal of draft t)
+ *   p_out   fp32 [batch, window, V]  this round's probabilities (rows 0..n-1 of each live image written)
+ *   cursor int32 [batch], seq int32 [batch, T+1], delta uint8 [batch, T+1], qbase int32 [batch]: rollout
+ *           state as in hbsjd_get_state, updated in place;  m_out int32 [batch]: tokens committed (images
+ *           with cursor == T are skipped and keep their m_out entry)
+ * The random words are Philox(seed; image, position, round).  Uses scratch buffers of the context; runs on
+ * the context's stream and waits for completion.  Limits: batch <= max_batch and window <= max_window of the
+ * context, V % 4 == 0, V <= 32768. */
+typedef struct {
+    int32_t batch, window, T, V, branches, history_offset, greedy, top_k;
+    float cfg_scale, temperature;
+    uint64_t seed;
+    uint32_t round;
+    uint32_t reserved;
+} hbsjd_verify_desc;
+int hbsjd_verify(hbsjd_ctx *c, const hbsjd_verify_desc *d, const float *logits, const float *q_prev, float *p_out,
+                 int32_t *cursor, int32_t *seq, uint8_t *delta, int32_t *qbase, int32_t *m_out);
+
 /* Per-kernel-class timing with CUDA events on the context's stream (off by default).  While enabled,
  * every launch of a timed class is bracketed by an event pair; totals accumulate until the next
  * hbsjd_profile(c, 1), which also resets them.  work = algorithmic FLOPs (GEMM: 2 M N K per launch) or

@@ -16,7 +16,7 @@ VERIFY_PROB, VERIFY_GREEDY = 0, 1
 EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
-EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
+EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
            "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_strerror", "hbsjd_last_error"]
 
 
@@ -50,6 +50,13 @@ class hbsjd_kernel_profile(C.Structure):
 PROF_CLASSES = ("gemm", "attention", "accept", "other")
 
 
+class hbsjd_verify_desc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("batch", "window", "T", "V", "branches", "history_offset", "greedy", "top_k")] + [
+                   ("cfg_scale", C.c_float), ("temperature", C.c_float), ("seed", C.c_uint64),
+                   ("round", C.c_uint32), ("reserved", C.c_uint32)]
+
+
 class HbsjdError(RuntimeError):
     def __init__(self, code, what, detail=""):
         super().__init__(f"{what}: {code} ({detail})")
@@ -74,6 +81,7 @@ def load():
         L.hbsjd_profile.argtypes = [vp, C.c_int]
         L.hbsjd_profile_read.argtypes = [vp, C.POINTER(hbsjd_kernel_profile)]
         L.hbsjd_probs.argtypes = [vp, vp, vp, C.c_int, C.c_float, C.c_float, C.c_int, vp]
+        L.hbsjd_verify.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
         L.hbsjd_round.argtypes = [vp, C.POINTER(C.c_int)]
         L.hbsjd_tokens.argtypes = [vp, vp]
         L.hbsjd_destroy.argtypes = [vp]
@@ -173,6 +181,12 @@ class Context:
                                          logits_c.shape[0], cfg_scale, temperature, top_k, out.data_ptr()),
                     "hbsjd_probs")
         return out
+
+    def hbsjd_verify(self, desc: hbsjd_verify_desc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out):
+        """Verification step on device tensors; state tensors are updated in place."""
+        self._check(self.lib.hbsjd_verify(self.h, C.byref(desc), logits.data_ptr(), q_prev.data_ptr(),
+                                          p_out.data_ptr(), cursor.data_ptr(), seq.data_ptr(), delta.data_ptr(),
+                                          qbase.data_ptr(), m_out.data_ptr()), "hbsjd_verify")
 
     def hbsjd_round(self) -> int:
         live = C.c_int(0)

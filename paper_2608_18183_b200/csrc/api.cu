@@ -55,6 +55,7 @@ struct hbsjd_ctx {
     long long launches;
     // host-buffer staging
     int32_t *stage_tok, *stage_len, *stage_lab, *stage_out;
+    void* verify_scratch;
     // per-class event timing
     bool profiling;
     struct ProfSlot { cudaEvent_t a, b; int cls; double work; };
@@ -316,7 +317,7 @@ void free_all(hbsjd_ctx* c) {
                     c->st.qbase, c->st.label, c->st.klen, c->st.pfill, c->st.slot_img, c->st.slot_c, c->st.slot_n,
                     c->st.counters, c->st.m_last, c->st.j_last, c->pbuf[0], c->pbuf[1], c->flag, c->cand_rep,
                     c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act,
-                    c->stage_tok, c->stage_len, c->stage_lab, c->stage_out};
+                    c->stage_tok, c->stage_len, c->stage_lab, c->stage_out, c->verify_scratch};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->h_counters) cudaFreeHost(c->h_counters);
@@ -460,6 +461,11 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
     if ((rc = dev_alloc(c, &c->stage_tok, Bm * (size_t)c->T)) || (rc = dev_alloc(c, &c->stage_len, Bm)) ||
         (rc = dev_alloc(c, &c->stage_lab, Bm)) || (rc = dev_alloc(c, &c->stage_out, Bm * (size_t)c->T)))
         return rc;
+    {
+        unsigned char* vs = nullptr;
+        if ((rc = dev_alloc(c, &vs, verify_scratch_bytes(c->Bmax, c->Wmax)))) return rc;
+        c->verify_scratch = vs;
+    }
     c->pool.resize(1024);
     for (auto& s : c->pool) {
         s.a = s.b = nullptr;
@@ -674,6 +680,25 @@ int hbsjd_probs(hbsjd_ctx* c, const float* logits_c, const float* logits_u, int 
         return HBSJD_EINVAL;
     launch_probs(logits_c, logits_u, rows, c->d.vocab, cfg_scale, temperature, top_k, probs, c->stream);
     CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
+}
+
+int hbsjd_verify(hbsjd_ctx* c, const hbsjd_verify_desc* d, const float* logits, const float* q_prev, float* p_out,
+                 int32_t* cursor, int32_t* seq, uint8_t* delta, int32_t* qbase, int32_t* m_out) {
+    if (!c) return HBSJD_EINVAL;
+    if (!d || !logits || !q_prev || !p_out || !cursor || !seq || !delta || !qbase || !m_out || d->batch < 1 ||
+        d->batch > c->Bmax || d->window < 1 || d->window > c->Wmax || d->T < 1 || d->V < 4 || d->V % 4 ||
+        d->V > 32768 || (d->branches != 1 && d->branches != 2) || d->history_offset < 1 ||
+        !(d->temperature > 0.f) || d->top_k < 0) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_verify: argument out of range");
+        return HBSJD_EINVAL;
+    }
+    static_assert(sizeof(VerifyDesc) == sizeof(hbsjd_verify_desc), "descriptor layouts must agree");
+    VerifyDesc vd;
+    memcpy(&vd, d, sizeof(vd));
+    const VerifyScratch sc = verify_scratch_carve(c->verify_scratch, d->batch, d->window);
+    CK(verify_enqueue(vd, sc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out, c->stream));
     CK(cudaStreamSynchronize(c->stream));
     return HBSJD_OK;
 }

@@ -230,11 +230,8 @@ __global__ void __launch_bounds__(QB * HPC * 32) k_attention_mma(State st, int S
 template <int QB, int HPC>
 void launch_cfg(const State& st, int S, int layer, const bf16* q, KvView kv, bf16* out, cudaStream_t s) {
     constexpr int smem = STAGES * HPC * 2 * KB * DH * 2;
-    static bool configured = false;
-    if (!configured) {
-        cudaFuncSetAttribute(k_attention_mma<QB, HPC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        configured = true;
-    }
+    static int configured[64] = {0};
+    ensure_dynamic_smem(k_attention_mma<QB, HPC>, smem, configured);
     dim3 grid(st.nb * S, st.Hh / HPC);
     launch_k(k_attention_mma<QB, HPC>, dim3(grid), dim3(QB * HPC * 32), smem, s, st, S, layer, q, kv, out);
 }

@@ -39,6 +39,20 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
 }
 
+// Raises a kernel's dynamic shared-memory limit once per device (function attributes are per device).
+template <typename K>
+inline cudaError_t ensure_dynamic_smem(K kernel, int bytes, int (&configured)[64]) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    if (bytes > configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e != cudaSuccess) return e;
+        configured[dev] = bytes;
+    }
+    return cudaSuccess;
+}
+
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f<bf16>(bf16 v) { return __bfloat162float(v); }

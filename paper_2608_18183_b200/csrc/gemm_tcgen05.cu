@@ -446,13 +446,9 @@ bool make_map_c(CUtensorMap* map, const float* base, int rows, int N) {
 template <int BN, int EPI>
 cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
                    cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(k_gemm_tcgen05<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             Cfg<BN>::SMEM);
-        if (e != cudaSuccess) return e;
-        configured = true;
-    }
+    static int configured[64] = {0};
+    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<BN, EPI>, Cfg<BN>::SMEM, configured);
+    if (e0 != cudaSuccess) return e0;
     const int tiles = (g.N / BN) * ((g.M + BM - 1) / BM);
     const int grid = tiles < num_sms() ? tiles : num_sms();
     return launch_k(k_gemm_tcgen05<BN, EPI>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<BN>::SMEM, s, ma, mw, mc, g);

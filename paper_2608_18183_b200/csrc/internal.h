@@ -64,6 +64,25 @@ void launch_swiglu(const float* gu, TA* act, int M, int F, cudaStream_t s);
 template <typename TA>
 void launch_gemm_simt(const TA* A, const TA* W, float* C, int M, int N, int K, int accumulate, cudaStream_t s);
 
+// Scratch of the stand-alone verification step, carved from one allocation.
+struct VerifyScratch {
+    int32_t *slot_img, *slot_c, *slot_n, *j_last, *counters;
+    uint8_t* flag;
+    int32_t *cand_rep, *cand_ref;
+};
+size_t verify_scratch_bytes(int batch, int window);
+VerifyScratch verify_scratch_carve(void* base, int batch, int window);
+struct VerifyDesc {  // mirrors hbsjd_verify_desc
+    int32_t batch, window, T, V, branches, history_offset, greedy, top_k;
+    float cfg_scale, temperature;
+    uint64_t seed;
+    uint32_t round, reserved;
+};
+// Enqueues set-up, probability/accept and commit kernels on caller state with the given scratch.
+cudaError_t verify_enqueue(const VerifyDesc& d, const VerifyScratch& sc, const float* logits, const float* q_prev,
+                           float* p_out, int32_t* cursor, int32_t* seq, uint8_t* delta, int32_t* qbase,
+                           int32_t* m_out, cudaStream_t s);
+
 // ---- tensor-core ragged attention, bf16, head size 64 (attention_mma.cu)
 bool attention_mma_supported(const State& st, const KvView& kv);
 void launch_attention_mma(const State& st, int S, int layer, const bf16* q, KvView kv, bf16* out, cudaStream_t s);

@@ -1,5 +1,7 @@
 // Rollout-state kernels: state init, prefill bookkeeping, initial history windows, and the fused
 // probability pipeline + SJD verification (Eq. 5; greedy Eq. 4) + commit + draft refresh.
+#include <cstring>
+
 #include "internal.h"
 
 namespace hbsjd {
@@ -504,22 +506,16 @@ int accept_smem_bytes(int V) { return V * (int)sizeof(float) + (int)sizeof(AccSh
 
 void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
                   float* p, cudaStream_t s) {
-    static int configured_bytes = 0;
+    static int configured[64] = {0};
     const int bytes = accept_smem_bytes(V);
-    if (bytes > configured_bytes) {
-        cudaFuncSetAttribute(k_probs, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        configured_bytes = bytes;
-    }
+    ensure_dynamic_smem(k_probs, bytes, configured);
     launch_k(k_probs, dim3(rows), dim3(ACC_THREADS), bytes, s, lc, lu, V, cfg_scale, temperature, top_k, p);
 }
 
 void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
-    static int configured_bytes = 0;
+    static int configured[64] = {0};
     const int bytes = accept_smem_bytes(st.V);
-    if (bytes > configured_bytes) {
-        cudaFuncSetAttribute(k_prob_accept, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-        configured_bytes = bytes;
-    }
+    ensure_dynamic_smem(k_prob_accept, bytes, configured);
     dim3 grid(st.W, a.S);
     launch_k(k_prob_accept, dim3(grid), dim3(ACC_THREADS), accept_smem_bytes(st.V), s, st, a);
 }
@@ -585,6 +581,74 @@ __global__ void k_commit(State st, AcceptArgs a) {
 
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s) {
     launch_k(k_commit, dim3((a.S + 3) / 4), dim3(128), 0, s, st, a);
+}
+
+// ------------------------------------------------------------------ stand-alone verification step
+size_t verify_scratch_bytes(int batch, int window) {
+    const size_t b = (size_t)batch, bw = (size_t)batch * window;
+    return 4 * b * 4 + 8 * 4 + (bw + 255) / 256 * 256 + 2 * bw * 4;
+}
+
+VerifyScratch verify_scratch_carve(void* base, int batch, int window) {
+    const size_t b = (size_t)batch, bw = (size_t)batch * window;
+    VerifyScratch sc;
+    unsigned char* p = (unsigned char*)base;
+    sc.slot_img = (int32_t*)p; p += b * 4;
+    sc.slot_c = (int32_t*)p;   p += b * 4;
+    sc.slot_n = (int32_t*)p;   p += b * 4;
+    sc.j_last = (int32_t*)p;   p += b * 4;
+    sc.counters = (int32_t*)p; p += 8 * 4;
+    sc.flag = p;               p += (bw + 255) / 256 * 256;
+    sc.cand_rep = (int32_t*)p; p += bw * 4;
+    sc.cand_ref = (int32_t*)p;
+    return sc;
+}
+
+cudaError_t verify_enqueue(const VerifyDesc& d, const VerifyScratch& sc, const float* logits, const float* q_prev,
+                           float* p_out, int32_t* cursor, int32_t* seq, uint8_t* delta, int32_t* qbase,
+                           int32_t* m_out, cudaStream_t s) {
+    State st;
+    memset(&st, 0, sizeof(st));
+    st.B = d.batch;
+    st.T = d.T;
+    st.V = d.V;
+    st.Bmax = d.batch;
+    st.Wmax = d.window;  // caller arrays are [batch][window][V]
+    st.W = d.window;
+    st.H = d.history_offset;
+    st.nb = d.branches;
+    st.cursor = cursor;
+    st.seq = seq;
+    st.delta = delta;
+    st.qbase = qbase;
+    st.slot_img = sc.slot_img;
+    st.slot_c = sc.slot_c;
+    st.slot_n = sc.slot_n;
+    st.counters = sc.counters;
+    st.m_last = m_out;
+    st.j_last = sc.j_last;
+    AcceptArgs a;
+    a.logits = logits;
+    a.pcur = p_out;
+    a.pprev = q_prev;
+    a.flag = sc.flag;
+    a.cand_rep = sc.cand_rep;
+    a.cand_ref = sc.cand_ref;
+    a.S = d.batch;
+    a.cfg_scale = d.cfg_scale;
+    a.temperature = d.temperature;
+    a.top_k = d.top_k;
+    a.greedy = d.greedy;
+    a.seed_lo = (uint32_t)(d.seed & 0xffffffffu);
+    a.seed_hi = (uint32_t)(d.seed >> 32);
+    a.round = d.round;
+    // the commit counters accumulate with atomics: they must start at zero on every call
+    cudaError_t e = cudaMemsetAsync(sc.counters, 0, 8 * sizeof(int32_t), s);
+    if (e != cudaSuccess) return e;
+    launch_setup(st, 0, 0, s);
+    launch_prob_accept(st, a, s);
+    launch_commit(st, a, s);
+    return cudaGetLastError();
 }
 
 }  // namespace hbsjd

@@ -153,3 +153,46 @@ def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, ma
         rep["rounds"] += 1
     return rep
 
+
+
+def verify_case(seed, B=24, W=16, T=64, V=2048, H=8, branches=1, sigma=0.6, cfg_scale=1.0, top_k=0):
+    """Synthetic inputs of the stand-alone verification step with a paper-like mix of accepted and rejected
+    drafts: proposals q = softmax(l + sigma * noise) against targets p = softmax(l), sampled drafts drawn from
+    their q rows, the rest history drafts (point-mass proposals), ragged cursors incl. a finished image.
+    Returns a dict of numpy arrays."""
+    rng = np.random.default_rng(seed)
+    base = (rng.normal(size=(B, W, V)) * 2.5).astype(np.float32)
+    logits = np.stack([base] + ([(base * 0.5 + rng.normal(size=base.shape) * 1.0).astype(np.float32)]
+                                if branches == 2 else []))
+    noise = sigma * rng.normal(size=base.shape).astype(np.float32)
+    cursor = rng.integers(0, T - 1, size=B).astype(np.int32)
+    cursor[0], cursor[1], cursor[2], cursor[3] = T, T - 1, T - 3, 0  # finished, one token left, ragged, empty
+    seq = rng.integers(0, V, size=(B, T + 1)).astype(np.int32)
+    delta = np.zeros((B, T + 1), dtype=np.uint8)
+    qbase = np.zeros(B, dtype=np.int32)
+    q = np.zeros((B, W, V), dtype=np.float32)
+    for b in range(B):
+        c = int(cursor[b])
+        back = int(rng.integers(1, 4))          # tokens committed in the previous round
+        qbase[b] = max(0, c - back)
+        shift = c - int(qbase[b])               # proposal of window position i sits in row i + shift
+        qlog = np.roll(base[b] + noise[b], shift, axis=0).astype(np.float64)
+        qlog -= qlog.max(-1, keepdims=True)
+        e = np.exp(qlog)
+        q[b] = (e / e.sum(-1, keepdims=True)).astype(np.float32)
+        n = min(W, T - c)
+        for t in range(c + 1, c + n):
+            qi = t - qbase[b] - 1
+            if qi < W and rng.random() < 0.85:  # a sampled draft with a stored proposal
+                pq = q[b, qi].astype(np.float64)
+                seq[b, t] = rng.choice(V, p=pq / pq.sum())
+                delta[b, t] = 0
+            else:                               # a history draft
+                delta[b, t] = 1
+    return dict(logits=logits, q=q, cursor=cursor, seq=seq, delta=delta, qbase=qbase, B=B, W=W, T=T, V=V, H=H,
+                branches=branches, cfg_scale=cfg_scale, top_k=top_k)
+
+
+def verify_desc(case, seed, rnd, greedy=False):
+    return binding.hbsjd_verify_desc(case["B"], case["W"], case["T"], case["V"], case["branches"], case["H"],
+                                     1 if greedy else 0, case["top_k"], case["cfg_scale"], 1.0, seed, rnd, 0)
