@@ -191,6 +191,32 @@ typedef struct {
 int hbsjd_verify(hbsjd_ctx *c, const hbsjd_verify_desc *d, const float *logits, const float *q_prev, float *p_out,
                  int32_t *cursor, int32_t *seq, uint8_t *delta, int32_t *qbase, int32_t *m_out);
 
+/* hbsjd_verify for callers that must not allocate device memory.  (The paper has no counterpart of this
+ * entry point; it exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a training process whose framework has
+ * handed the whole device to its own caching allocator (a raw allocation there can fail or fragment the
+ * pool), a latency-critical loop in which an allocation would synchronise the device, or a plug-in called
+ * from inside another runtime that owns all device memory.  Such a caller cannot create an hbsjd_ctx either,
+ * so this function takes no context: it needs only the stream, the descriptor and the same input / output
+ * buffers as hbsjd_verify.
+ *
+ * How: the scratch of the verification kernels (slot tables, accept flags, candidate tokens, counters) lives
+ * in a fixed array of 192 KiB that is part of the library image; every GPU that loads the library holds it
+ * until the process exits.  The function calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Limits: batch <= 1024, batch * window <= 16384, window <= 64, V % 4 == 0, V <= 32768; larger requests
+ *     are refused with HBSJD_EINVAL and nothing is launched.
+ *   - The first call on each device looks up the array's device address and raises the kernels' shared-
+ *     memory limit; make that first call before any stream capture begins.
+ *   - Every call uses the same array and finds the previous call's contents in it; the function clears
+ *     what has to start at zero.  Calls that overlap on the GPU (other streams, other host threads) race on
+ *     the array: serialise them.
+ *   - cuda_stream is a cudaStream_t passed as void*; the call returns after the stream has finished the work.
+ * Results are identical to hbsjd_verify on the same inputs. */
+int hbsjd_verify_static(void *cuda_stream, const hbsjd_verify_desc *d, const float *logits, const float *q_prev,
+                        float *p_out, int32_t *cursor, int32_t *seq, uint8_t *delta, int32_t *qbase,
+                        int32_t *m_out);
+
 /* Per-kernel-class timing with CUDA events on the context's stream (off by default).  While enabled,
  * every launch of a timed class is bracketed by an event pair; totals accumulate until the next
  * hbsjd_profile(c, 1), which also resets them.  work = algorithmic FLOPs (GEMM: 2 M N K per launch) or

@@ -16,7 +16,7 @@ VERIFY_PROB, VERIFY_GREEDY = 0, 1
 EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
-EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
+EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
            "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_strerror", "hbsjd_last_error"]
 
 
@@ -82,6 +82,7 @@ def load():
         L.hbsjd_profile_read.argtypes = [vp, C.POINTER(hbsjd_kernel_profile)]
         L.hbsjd_probs.argtypes = [vp, vp, vp, C.c_int, C.c_float, C.c_float, C.c_int, vp]
         L.hbsjd_verify.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
+        L.hbsjd_verify_static.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
         L.hbsjd_round.argtypes = [vp, C.POINTER(C.c_int)]
         L.hbsjd_tokens.argtypes = [vp, vp]
         L.hbsjd_destroy.argtypes = [vp]
@@ -108,6 +109,16 @@ def make_params(window, history_offset, cfg_scale=1.0, temperature=1.0, top_k=0,
                 exec_mode=EXEC_HYBRID, gamma=0, seed=0, max_rounds=-1) -> hbsjd_params:
     return hbsjd_params(window, history_offset, cfg_scale, temperature, top_k, verify_mode, exec_mode, gamma, seed,
                         max_rounds, 0)
+
+
+def hbsjd_verify_static(stream, desc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out):
+    """The allocation-free verification step: no context, scratch inside the library image.
+    `stream` is a torch.cuda.Stream; tensors are device tensors, state updated in place."""
+    rc = load().hbsjd_verify_static(C.c_void_p(stream.cuda_stream), C.byref(desc), logits.data_ptr(),
+                                    q_prev.data_ptr(), p_out.data_ptr(), cursor.data_ptr(), seq.data_ptr(),
+                                    delta.data_ptr(), qbase.data_ptr(), m_out.data_ptr())
+    if rc != 0:
+        raise HbsjdError(rc, "hbsjd_verify_static", load().hbsjd_strerror(rc).decode())
 
 
 class Context:

@@ -1,7 +1,9 @@
 // Rollout-state kernels: state init, prefill bookkeeping, initial history windows, and the fused
 // probability pipeline + SJD verification (Eq. 5; greedy Eq. 4) + commit + draft refresh.
 #include <cstring>
+#include <mutex>
 
+#include "../../include/hbsjd.h"
 #include "internal.h"
 
 namespace hbsjd {
@@ -652,3 +654,51 @@ cudaError_t verify_enqueue(const VerifyDesc& d, const VerifyScratch& sc, const f
 }
 
 }  // namespace hbsjd
+
+// ------------------------------------------------------------------ verification without any allocation
+// Scratch for callers that may not allocate: a fixed device array inside the library image.  In host code
+// the symbol below is only a handle; the device address is looked up once per device with
+// cudaGetSymbolAddress (that device current) and handed to the kernels as an ordinary pointer.
+namespace {
+constexpr size_t kStaticScratchBytes = 192 * 1024;
+static __device__ __align__(256) unsigned char g_verify_scratch[kStaticScratchBytes];
+
+std::mutex g_static_mu;
+void* g_static_ptr[64] = {nullptr};
+}  // namespace
+
+extern "C" int hbsjd_verify_static(void* cuda_stream, const hbsjd_verify_desc* d, const float* logits,
+                                   const float* q_prev, float* p_out, int32_t* cursor, int32_t* seq, uint8_t* delta,
+                                   int32_t* qbase, int32_t* m_out) {
+    using namespace hbsjd;
+    if (!d || !logits || !q_prev || !p_out || !cursor || !seq || !delta || !qbase || !m_out) return HBSJD_EINVAL;
+    if (d->batch < 1 || d->batch > 1024 || d->window < 1 || d->window > 64 ||
+        (long)d->batch * d->window > 16384 || d->T < 1 || d->V < 4 || d->V % 4 || d->V > 32768 ||
+        (d->branches != 1 && d->branches != 2) || d->history_offset < 1 || !(d->temperature > 0.f) || d->top_k < 0)
+        return HBSJD_EINVAL;
+    if (verify_scratch_bytes(d->batch, d->window) > kStaticScratchBytes) return HBSJD_EINVAL;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HBSJD_ECUDA;
+    void* base = nullptr;
+    {
+        // once per device: the array's address on the current device
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_verify_scratch) != cudaSuccess || !ptr) return HBSJD_ECUDA;
+            g_static_ptr[dev] = ptr;
+        }
+        base = g_static_ptr[dev];
+    }
+    static_assert(sizeof(VerifyDesc) == sizeof(hbsjd_verify_desc), "descriptor layouts must agree");
+    VerifyDesc vd;
+    memcpy(&vd, d, sizeof(vd));
+    const VerifyScratch sc = verify_scratch_carve(base, d->batch, d->window);
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // verify_enqueue zeroes the counters; the slot tables, flags and candidates are fully rewritten for
+    // every (image, position) that is read back, so stale contents of the previous call are never used
+    if (verify_enqueue(vd, sc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out, s) != cudaSuccess)
+        return HBSJD_ECUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return HBSJD_ECUDA;
+    return HBSJD_OK;
+}
