@@ -107,10 +107,14 @@ void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s) {
 constexpr int ACC_THREADS = 512;
 constexpr int ACC_WARPS = ACC_THREADS / 32;
 
+// Work area + reduction scratch behind the V floats.  Sized so that three CTAs fit one SM at V = 16384.
+constexpr int SEL_BINS = 1024;
+constexpr int SEL_CAP = 1536;
 struct AccShared {
-    unsigned int hist[ACC_WARPS][256];
+    unsigned int work[SEL_BINS + SEL_CAP];  // selection histogram, then the keys of the selected bin
     float redf[ACC_WARPS];
-    unsigned long long redu[ACC_WARPS];
+    float red4[4][ACC_WARPS];                // min / max / sum / sum of squares per warp
+    unsigned long long redu[ACC_WARPS];      // per-warp sums of the fixed-point weights of the current array
     unsigned int sel_prefix, sel_k;
     int result;
     uint32_t words[4];
@@ -146,46 +150,50 @@ __device__ __forceinline__ float block_sum(float v, AccShared& sh) {
 
 __device__ __forceinline__ unsigned int fixed_weight(float a) { return __float2uint_rd(a * 1073741824.0f); }
 
-// Fixed-point categorical sample over a[0..V) in shared memory (all threads call).  -1 if the total is 0.
-__device__ int block_sample(const float* a, int V, uint32_t word, AccShared& sh) {
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int seg = (((V + ACC_WARPS - 1) / ACC_WARPS) + 31) / 32 * 32;
-    const int base = wid * seg;
-    unsigned long long part = 0;
-    for (int it = 0; it < seg; it += 32) {
-        const int v = base + it + lane;
-        if (v < V) part += fixed_weight(a[v]);
-    }
+// Warp w owns the contiguous segment [w * seg, (w+1) * seg) of the vocabulary (seg a multiple of 128).
+__device__ __forceinline__ int warp_segment(int V) { return (((V + ACC_WARPS - 1) / ACC_WARPS) + 127) / 128 * 128; }
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
-    __syncthreads();
-    if (lane == 0) sh.redu[wid] = part;
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Fixed-point categorical pick over a[0..V) (shared memory) whose per-warp weight sums are in sh.redu
+// (all threads call; ends with a barrier).  Integer running sums: the result is the smallest v whose
+// inclusive sum exceeds (word * S) >> 32, whatever the order of evaluation.  -1 if the total is 0.
+__device__ int block_pick(const float* a, int V, uint32_t word, AccShared& sh) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int seg = warp_segment(V);
+    const int base = wid * seg;
     if (threadIdx.x == 0) sh.result = -1;
     __syncthreads();
-    unsigned long long S = 0;
+    unsigned long long S = 0, excl = 0;
 #pragma unroll
-    for (int w = 0; w < ACC_WARPS; ++w) S += sh.redu[w];
-    if (S == 0) return -1;
-    const unsigned long long target = ((unsigned long long)word * S) >> 32;
-    unsigned long long excl = 0;
-    for (int w = 0; w < wid; ++w) excl += sh.redu[w];
-    if (target >= excl && target < excl + sh.redu[wid]) {  // exactly one warp
-        unsigned long long run = excl;
-        for (int it = 0; it < seg; it += 32) {
-            const int v = base + it + lane;
-            unsigned long long x = (v < V) ? fixed_weight(a[v]) : 0ull;
-            unsigned long long incl = x;
+    for (int w = 0; w < ACC_WARPS; ++w) {
+        if (w == wid) excl = S;
+        S += sh.redu[w];
+    }
+    if (S != 0) {
+        const unsigned long long target = ((unsigned long long)word * S) >> 32;
+        if (target >= excl && target < excl + sh.redu[wid]) {  // exactly one warp
+            unsigned long long run = excl;
+            for (int it = 0; it < seg; it += 32) {
+                const int v = base + it + lane;
+                const unsigned long long x = (v < V) ? fixed_weight(a[v]) : 0ull;
+                unsigned long long incl = x;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += t;
+                }
+                const unsigned int hit = __ballot_sync(0xffffffffu, run + incl > target);
+                if (hit) {
+                    if (lane == 0) sh.result = base + it + (__ffs(hit) - 1);
+                    break;
+                }
+                run += __shfl_sync(0xffffffffu, incl, 31);
             }
-            const unsigned int hit = __ballot_sync(0xffffffffu, run + incl > target);
-            if (hit) {
-                if (lane == 0) sh.result = base + it + (__ffs(hit) - 1);
-                break;
-            }
-            run += __shfl_sync(0xffffffffu, incl, 31);
         }
     }
     __syncthreads();
@@ -195,6 +203,7 @@ __device__ int block_sample(const float* a, int V, uint32_t word, AccShared& sh)
 // Key of the k-th largest of g[0..V) by radix select, one byte per pass from the top (exact for any input).
 __device__ unsigned int radix_select(const float* g, int V, unsigned int k, AccShared& sh) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    unsigned int* hist = sh.work;  // [256]
     if (tid == 0) {
         sh.sel_prefix = 0u;
         sh.sel_k = k;
@@ -202,12 +211,12 @@ __device__ unsigned int radix_select(const float* g, int V, unsigned int k, AccS
     for (int pass = 0; pass < 4; ++pass) {
         const int shift = 24 - 8 * pass;
         const unsigned int mask = pass == 0 ? 0u : (0xFFFFFFFFu << (shift + 8));
-        for (int x = lane; x < 256; x += 32) sh.hist[wid][x] = 0u;
+        for (int x = tid; x < 256; x += ACC_THREADS) hist[x] = 0u;
         __syncthreads();
         const unsigned int prefix = sh.sel_prefix;
         for (int v = tid; v < V; v += ACC_THREADS) {
             const unsigned int key = float_key(g[v]);
-            if ((key & mask) == prefix) atomicAdd(&sh.hist[wid][(key >> shift) & 255u], 1u);
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
         if (wid == 0) {
@@ -215,10 +224,8 @@ __device__ unsigned int radix_select(const float* g, int V, unsigned int k, AccS
             unsigned int cnt[8], tot = 0;
 #pragma unroll
             for (int x = 0; x < 8; ++x) {
-                unsigned int s = 0;
-                for (int w = 0; w < ACC_WARPS; ++w) s += sh.hist[w][lane * 8 + x];
-                cnt[x] = s;
-                tot += s;
+                cnt[x] = hist[lane * 8 + x];
+                tot += cnt[x];
             }
             unsigned int incl = tot;
 #pragma unroll
@@ -246,141 +253,237 @@ __device__ unsigned int radix_select(const float* g, int V, unsigned int k, AccS
     return sh.sel_prefix;
 }
 
-// Key of the k-th largest of g[0..V), 0 < k < V.  One pass builds a 1024-bin histogram over [min, max]
-// with a monotone binning (a higher bin holds strictly larger values), which locates the bin of the k-th
-// largest and its rank inside that bin; the few entries of that bin are then ranked exactly against one
-// another.  Falls back to the radix select when that bin is crowded.  *gmax receives max(g).
-constexpr int SEL_BINS = 1024;
-constexpr int SEL_CAP = 2048;
-__device__ unsigned int topk_threshold(const float* g, int V, unsigned int k, AccShared& sh, float* gmax) {
+// Key of the k-th largest of g[0..V), 0 < k < V, given mn = min(g), mx = max(g) and a guess `lo` of a value
+// below it (any lo <= mx is safe: a wrong guess only costs a second pass).  One pass builds a 1024-bin
+// histogram of the entries >= lo over [lo, mx] with a monotone binning (a higher bin holds strictly larger
+// values), which locates the bin of the k-th largest and its rank inside that bin; the few entries of that
+// bin are then ranked exactly against one another.  If fewer than k entries lie above lo the pass is
+// repeated over [mn, mx]; a crowded bin falls back to the radix select.
+__device__ unsigned int topk_threshold(const float* g, int V, unsigned int k, float mn, float mx, float lo,
+                                       AccShared& sh) {
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    unsigned int* hist = &sh.hist[0][0];       // [SEL_BINS]
-    unsigned int* cand = hist + SEL_BINS;      // [SEL_CAP] keys of the entries of the selected bin
-    float mn = INFINITY, mx = -INFINITY;
-    for (int v = tid; v < V; v += ACC_THREADS) {
-        const float x = g[v];
-        mn = fminf(mn, x);
-        mx = fmaxf(mx, x);
-    }
-    mx = block_max(mx, sh);
-    mn = -block_max(-mn, sh);
-    *gmax = mx;
-    if (!(mx > mn)) return float_key(mn);  // all entries equal: everything is kept
-    const float scale = (float)SEL_BINS / (mx - mn);
-    for (int x = tid; x < SEL_BINS; x += ACC_THREADS) hist[x] = 0u;
-    if (tid == 0) {
-        sh.sel_prefix = 0u;  // selected bin
-        sh.sel_k = 0u;       // rank of the k-th largest inside it (1-based, from the top)
-        sh.result = 0;       // candidate count
-    }
-    __syncthreads();
-    for (int v = tid; v < V; v += ACC_THREADS) {
-        const int b = min(SEL_BINS - 1, (int)((g[v] - mn) * scale));
-        atomicAdd(&hist[b], 1u);
-    }
-    __syncthreads();
-    if (wid == 0) {
-        unsigned int tot = 0;
-        for (int x = 0; x < 32; ++x) tot += hist[lane * 32 + x];
-        unsigned int incl = tot;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned int tt = __shfl_down_sync(0xffffffffu, incl, o);
-            if (lane + o < 32) incl += tt;
+
+    unsigned int* hist = sh.work;             // [SEL_BINS]
+    unsigned int* cand = sh.work + SEL_BINS;  // [SEL_CAP] keys of the entries of the selected bin
+    if (!(mx > mn)) return float_key(mn);     // all entries equal: everything is kept
+    if (!(lo > mn) || !(lo < mx)) lo = mn;
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        const float scale = (float)SEL_BINS / (mx - lo);
+        for (int x = tid; x < SEL_BINS; x += ACC_THREADS) hist[x] = 0u;
+        if (tid == 0) {
+            sh.sel_prefix = 0xFFFFFFFFu;  // selected bin (none yet)
+            sh.sel_k = 0u;                // rank of the k-th largest inside it (1-based, from the top)
+            sh.result = 0;                // candidate count
         }
-        unsigned int above = incl - tot;
-        if (above < k && k <= above + tot) {  // exactly one lane
-            for (int x = 31; x >= 0; --x) {
-                const unsigned int c = hist[lane * 32 + x];
-                if (k <= above + c) {
-                    sh.sel_prefix = (unsigned int)(lane * 32 + x);
-                    sh.sel_k = k - above;
-                    break;
+        __syncthreads();
+        for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+            const float4 x = *reinterpret_cast<const float4*>(g + v);
+            if (x.x >= lo) atomicAdd(&hist[min(SEL_BINS - 1, (int)((x.x - lo) * scale))], 1u);
+            if (x.y >= lo) atomicAdd(&hist[min(SEL_BINS - 1, (int)((x.y - lo) * scale))], 1u);
+            if (x.z >= lo) atomicAdd(&hist[min(SEL_BINS - 1, (int)((x.z - lo) * scale))], 1u);
+            if (x.w >= lo) atomicAdd(&hist[min(SEL_BINS - 1, (int)((x.w - lo) * scale))], 1u);
+        }
+        __syncthreads();
+        if (wid == 0) {
+            unsigned int tot = 0;
+            for (int x = 0; x < 32; ++x) tot += hist[lane * 32 + ((x + lane) & 31)];  // rotated: no bank conflict
+            unsigned int incl = tot;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int tt = __shfl_down_sync(0xffffffffu, incl, o);
+                if (lane + o < 32) incl += tt;
+            }
+            unsigned int above = incl - tot;
+            if (above < k && k <= above + tot) {  // at most one lane; none if fewer than k entries are >= lo
+                for (int x = 31; x >= 0; --x) {
+                    const unsigned int c = hist[lane * 32 + x];
+                    if (k <= above + c) {
+                        sh.sel_prefix = (unsigned int)(lane * 32 + x);
+                        sh.sel_k = k - above;
+                        break;
+                    }
+                    above += c;
                 }
-                above += c;
             }
         }
-    }
-    __syncthreads();
-    const int bsel = (int)sh.sel_prefix;
-    const unsigned int krem = sh.sel_k;
-    for (int v = tid; v < V; v += ACC_THREADS) {
-        const float x = g[v];
-        if (min(SEL_BINS - 1, (int)((x - mn) * scale)) == bsel) {
-            const int slot = atomicAdd(&sh.result, 1);
-            if (slot < SEL_CAP) cand[slot] = float_key(x);
+        __syncthreads();
+        const unsigned int bsel = sh.sel_prefix;
+        const unsigned int krem = sh.sel_k;
+        if (bsel == 0xFFFFFFFFu) {  // the guess was too high: histogram the whole range
+            __syncthreads();
+            lo = mn;
+            continue;
         }
-    }
-    __syncthreads();
-    const int nc = sh.result;
-    __syncthreads();
-    if (nc > SEL_CAP) return radix_select(g, V, k, sh);
-    // the value with (#strictly greater) < krem <= (#greater or equal) is the krem-th largest of the bin
-    for (int i = tid; i < nc; i += ACC_THREADS) {
-        const unsigned int ki = cand[i];
-        unsigned int gt = 0, ge = 0;
-        for (int j = 0; j < nc; ++j) {
-            const unsigned int kj = cand[j];
-            gt += kj > ki;
-            ge += kj >= ki;
+        for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+            const float4 x4 = *reinterpret_cast<const float4*>(g + v);
+            const float xs[4] = {x4.x, x4.y, x4.z, x4.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float x = xs[e];
+                if (x >= lo && min(SEL_BINS - 1, (int)((x - lo) * scale)) == (int)bsel) {
+                    const int slot = atomicAdd(&sh.result, 1);
+                    if (slot < SEL_CAP) cand[slot] = float_key(x);
+                }
+            }
         }
-        if (gt < krem && krem <= ge) sh.sel_prefix = ki;  // every such thread writes the same key
+        __syncthreads();
+        const int nc = sh.result;
+        __syncthreads();
+        if (nc > SEL_CAP) return radix_select(g, V, k, sh);
+        // the value with (#strictly greater) < krem <= (#greater or equal) is the krem-th largest of the bin
+        for (int i = tid; i < nc; i += ACC_THREADS) {
+            const unsigned int ki = cand[i];
+            unsigned int gt = 0, ge = 0;
+            for (int j = 0; j < nc; ++j) {
+                const unsigned int kj = cand[j];
+                gt += kj > ki;
+                ge += kj >= ki;
+            }
+            if (gt < krem && krem <= ge) sh.sel_prefix = ki;  // every such thread writes the same key
+        }
+        __syncthreads();
+        const unsigned int theta = sh.sel_prefix;
+        __syncthreads();
+        return theta;
+    }
+    return radix_select(g, V, k, sh);  // not reached: the second attempt covers every entry
+}
+
+// Block-wide min, max, sum and sum of squares (two barriers).
+__device__ void block_stats(float& mn, float& mx, float& s1, float& s2, AccShared& sh) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        s1 += __shfl_xor_sync(0xffffffffu, s1, o);
+        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
     }
     __syncthreads();
-    const unsigned int theta = sh.sel_prefix;
+    if (lane == 0) {
+        sh.red4[0][wid] = mn;
+        sh.red4[1][wid] = mx;
+        sh.red4[2][wid] = s1;
+        sh.red4[3][wid] = s2;
+    }
     __syncthreads();
-    return theta;
+    mn = sh.red4[0][0];
+    mx = sh.red4[1][0];
+    s1 = sh.red4[2][0];
+    s2 = sh.red4[3][0];
+#pragma unroll
+    for (int w = 1; w < ACC_WARPS; ++w) {
+        mn = fminf(mn, sh.red4[0][w]);
+        mx = fmaxf(mx, sh.red4[1][w]);
+        s1 += sh.red4[2][w];
+        s2 += sh.red4[3][w];
+    }
 }
 
 // Probability pipeline of one position, all threads of the CTA: guided = l_u + s (l_c - l_u); divided by
-// the temperature; top-k threshold (ties kept); softmax in fp32.  Leaves p in g[0..V) (shared memory) and
-// writes it to pout.  Ends with a block-wide barrier.
+// the temperature; top-k threshold (ties kept); softmax in fp32.  Leaves p in g[0..V) (shared memory),
+// writes it to pout, and leaves the per-warp fixed-point weight sums of p in sh.redu.  Ends with a barrier.
 __device__ void prob_pipeline(float* g, const float* __restrict__ lc, const float* __restrict__ lu, int V,
                               float cfg_scale, float temperature, int top_k, float* __restrict__ pout,
                               AccShared& sh) {
-    const int tid = threadIdx.x;
-    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
-        float4 x = *reinterpret_cast<const float4*>(lc + v);
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    float mn = INFINITY, mx = -INFINITY, s1 = 0.f, s2 = 0.f;
+    const bool select = top_k > 0 && top_k < V;
+    // The conditional logits go straight to shared memory with cp.async (every copy of the row in flight
+    // at once); the unconditional ones are fetched eight float4 at a time into registers meanwhile.  A
+    // thread combines exactly the elements it copied, so waiting for its own copies is enough.
+    const uint32_t g_s = (uint32_t)__cvta_generic_to_shared(g);
+    for (int v = tid * 4; v < V; v += ACC_THREADS * 4)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(g_s + (uint32_t)v * 4u), "l"(lc + v)
+                     : "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int v0 = tid * 4; v0 < V; v0 += ACC_THREADS * 4 * 8) {
+        float4 y[8];
         if (lu) {
-            const float4 y = *reinterpret_cast<const float4*>(lu + v);
-            x.x = __fadd_rn(y.x, __fmul_rn(cfg_scale, __fsub_rn(x.x, y.x)));
-            x.y = __fadd_rn(y.y, __fmul_rn(cfg_scale, __fsub_rn(x.y, y.y)));
-            x.z = __fadd_rn(y.z, __fmul_rn(cfg_scale, __fsub_rn(x.z, y.z)));
-            x.w = __fadd_rn(y.w, __fmul_rn(cfg_scale, __fsub_rn(x.w, y.w)));
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const int v = v0 + k * ACC_THREADS * 4;
+                if (v < V) y[k] = *reinterpret_cast<const float4*>(lu + v);
+            }
         }
-        x.x = __fdiv_rn(x.x, temperature);
-        x.y = __fdiv_rn(x.y, temperature);
-        x.z = __fdiv_rn(x.z, temperature);
-        x.w = __fdiv_rn(x.w, temperature);
-        *reinterpret_cast<float4*>(g + v) = x;
+        if (v0 == tid * 4) asm volatile("cp.async.wait_all;" ::: "memory");
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int v = v0 + k * ACC_THREADS * 4;
+            if (v < V) {
+                float4 x = *reinterpret_cast<float4*>(g + v);
+                if (lu) {
+                    x.x = __fadd_rn(y[k].x, __fmul_rn(cfg_scale, __fsub_rn(x.x, y[k].x)));
+                    x.y = __fadd_rn(y[k].y, __fmul_rn(cfg_scale, __fsub_rn(x.y, y[k].y)));
+                    x.z = __fadd_rn(y[k].z, __fmul_rn(cfg_scale, __fsub_rn(x.z, y[k].z)));
+                    x.w = __fadd_rn(y[k].w, __fmul_rn(cfg_scale, __fsub_rn(x.w, y[k].w)));
+                }
+                if (temperature != 1.0f) {
+                    x.x = __fdiv_rn(x.x, temperature);
+                    x.y = __fdiv_rn(x.y, temperature);
+                    x.z = __fdiv_rn(x.z, temperature);
+                    x.w = __fdiv_rn(x.w, temperature);
+                }
+                *reinterpret_cast<float4*>(g + v) = x;
+                mn = fminf(fminf(mn, x.x), fminf(fminf(x.y, x.z), x.w));
+                mx = fmaxf(fmaxf(mx, x.x), fmaxf(fmaxf(x.y, x.z), x.w));
+                if (select) {
+                    s1 += (x.x + x.y) + (x.z + x.w);
+                    s2 += (x.x * x.x + x.y * x.y) + (x.z * x.z + x.w * x.w);
+                }
+            }
+        }
     }
-    __syncthreads();
     unsigned int theta = 0u;
-    float mx;
-    if (top_k > 0 && top_k < V) {
-        theta = topk_threshold(g, V, (unsigned int)top_k, sh, &mx);  // the largest entry is always kept
+    if (select) {
+        block_stats(mn, mx, s1, s2, sh);  // the barriers inside also publish g
+        // Guess a value below the k-th largest from a normal fit of the row: the upper-tail quantile of
+        // 1.5 k / V (+ a small absolute margin), by the rational approximation of Abramowitz & Stegun
+        // 26.2.23.  Only entries above the guess enter the selection histogram; the guess is verified by
+        // the count and costs a second pass if it was too high.
+        const float mean = s1 / (float)V;
+        const float sd = sqrtf(fmaxf(s2 / (float)V - mean * mean, 0.f));
+        const float f = fminf(0.5f, (1.5f * (float)top_k + 16.f) / (float)V);
+        const float tq = sqrtf(-2.0f * __logf(f));
+        const float zq = tq - (2.515517f + tq * (0.802853f + tq * 0.010328f)) /
+                                  (1.0f + tq * (1.432788f + tq * (0.189269f + tq * 0.001308f)));
+        theta = topk_threshold(g, V, (unsigned int)top_k, mn, mx, mean + zq * sd, sh);
     } else {
-        mx = -INFINITY;
-        for (int v = tid; v < V; v += ACC_THREADS) mx = fmaxf(mx, g[v]);
-        mx = block_max(mx, sh);
+        mx = block_max(mx, sh);  // the barriers inside also publish g
     }
+    // exp and normalisation.  The threshold key is turned back into the float it encodes, so "kept" is one
+    // float compare; ex2.approx (relative error about 1e-6 over the range used) and a multiplication by
+    // 1/sum replace expf and the division: both sit well inside the probability tolerance, and every
+    // downstream decision uses these very numbers.
+    const float thr = theta == 0u ? -INFINITY
+                                  : __uint_as_float((theta & 0x80000000u) ? (theta & 0x7FFFFFFFu) : ~theta);
     float part = 0.f;
-    for (int v = tid; v < V; v += ACC_THREADS) {
-        const float x = g[v];
-        const float e = float_key(x) >= theta ? expf(x - mx) : 0.f;
-        g[v] = e;
-        part += e;
+    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+        float4 x = *reinterpret_cast<float4*>(g + v);
+        x.x = x.x >= thr ? __expf(x.x - mx) : 0.f;
+        x.y = x.y >= thr ? __expf(x.y - mx) : 0.f;
+        x.z = x.z >= thr ? __expf(x.z - mx) : 0.f;
+        x.w = x.w >= thr ? __expf(x.w - mx) : 0.f;
+        *reinterpret_cast<float4*>(g + v) = x;
+        part += (x.x + x.y) + (x.z + x.w);
     }
     const float den = block_sum(part, sh);
-    for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
+    const float inv = 1.0f / den;
+    // normalise segment-wise (warp w owns [w*seg, (w+1)*seg)) so that the sampler's per-warp sums fall out
+    const int seg = warp_segment(V);
+    unsigned long long wsum = 0;
+    for (int v = wid * seg + lane * 4; v < min(V, (wid + 1) * seg); v += 128) {
         float4 e = *reinterpret_cast<float4*>(g + v);
-        e.x = __fdiv_rn(e.x, den);
-        e.y = __fdiv_rn(e.y, den);
-        e.z = __fdiv_rn(e.z, den);
-        e.w = __fdiv_rn(e.w, den);
+        e.x *= inv;
+        e.y *= inv;
+        e.z *= inv;
+        e.w *= inv;
         *reinterpret_cast<float4*>(g + v) = e;
         *reinterpret_cast<float4*>(pout + v) = e;
+        wsum += (unsigned long long)fixed_weight(e.x) + fixed_weight(e.y) + fixed_weight(e.z) + fixed_weight(e.w);
     }
+    wsum = warp_sum_u64(wsum);
+    if (lane == 0) sh.redu[wid] = wsum;
     __syncthreads();
 }
 
@@ -468,34 +571,59 @@ __global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArg
     }
     const uint32_t w1 = sh.words[1], w2 = sh.words[2];
 
-    // refreshed draft candidate ~ p_i
-    const int ref = block_sample(g, V, w2, sh);
+    // refreshed draft candidate ~ p_i (weight sums already in sh.redu)
+    const int ref = block_pick(g, V, w2, sh);
     int rep = -1;
     if (last) {
-        rep = block_sample(g, V, w1, sh);  // bonus token ~ p_{n-1}
+        rep = block_pick(g, V, w1, sh);  // bonus token ~ p_{n-1}: same array, same sums
     } else if (!accept) {
         // residual [p - q]+ (point-mass proposal: p with z removed), overwriting p in shared memory
+        const int seg = warp_segment(V);
         if (is_delta) {
-            if (tid == 0) g[z] = 0.f;
-        } else {
-            for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
-                float4 p4 = *reinterpret_cast<float4*>(g + v);
-                const float4 q4 = *reinterpret_cast<const float4*>(qrow + v);
-                p4.x = fmaxf(__fsub_rn(p4.x, q4.x), 0.f);
-                p4.y = fmaxf(__fsub_rn(p4.y, q4.y), 0.f);
-                p4.z = fmaxf(__fsub_rn(p4.z, q4.z), 0.f);
-                p4.w = fmaxf(__fsub_rn(p4.w, q4.w), 0.f);
-                *reinterpret_cast<float4*>(g + v) = p4;
+            if (tid == 0) {
+                sh.redu[z / seg] -= fixed_weight(g[z]);
+                g[z] = 0.f;
             }
+        } else {
+            unsigned long long wsum = 0;
+            const int vend = min(V, (wid + 1) * seg);
+            for (int v0 = wid * seg + lane * 4; v0 < vend; v0 += 128 * 8) {
+                float4 q4[8];  // eight proposal loads in flight per thread
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (v0 + k * 128 < vend) q4[k] = *reinterpret_cast<const float4*>(qrow + v0 + k * 128);
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const int v = v0 + k * 128;
+                    if (v < vend) {
+                        float4 p4 = *reinterpret_cast<float4*>(g + v);
+                        p4.x = fmaxf(__fsub_rn(p4.x, q4[k].x), 0.f);
+                        p4.y = fmaxf(__fsub_rn(p4.y, q4[k].y), 0.f);
+                        p4.z = fmaxf(__fsub_rn(p4.z, q4[k].z), 0.f);
+                        p4.w = fmaxf(__fsub_rn(p4.w, q4[k].w), 0.f);
+                        *reinterpret_cast<float4*>(g + v) = p4;
+                        wsum += (unsigned long long)fixed_weight(p4.x) + fixed_weight(p4.y) + fixed_weight(p4.z) +
+                                fixed_weight(p4.w);
+                    }
+                }
+            }
+            wsum = warp_sum_u64(wsum);
+            if (lane == 0) sh.redu[wid] = wsum;
         }
         __syncthreads();
-        rep = block_sample(g, V, w1, sh);
+        rep = block_pick(g, V, w1, sh);
         if (rep < 0) {  // empty residual: sample p_i itself with the same word
+            unsigned long long wsum = 0;
+            for (int v = wid * seg + lane * 4; v < min(V, (wid + 1) * seg); v += 128) {
+                const float4 p4 = *reinterpret_cast<const float4*>(pout + v);
+                *reinterpret_cast<float4*>(g + v) = p4;
+                wsum += (unsigned long long)fixed_weight(p4.x) + fixed_weight(p4.y) + fixed_weight(p4.z) +
+                        fixed_weight(p4.w);
+            }
+            wsum = warp_sum_u64(wsum);
+            if (lane == 0) sh.redu[wid] = wsum;
             __syncthreads();
-            for (int v = tid * 4; v < V; v += ACC_THREADS * 4)
-                *reinterpret_cast<float4*>(g + v) = *reinterpret_cast<const float4*>(pout + v);
-            __syncthreads();
-            rep = block_sample(g, V, w1, sh);
+            rep = block_pick(g, V, w1, sh);
         }
     }
     if (tid == 0) {
