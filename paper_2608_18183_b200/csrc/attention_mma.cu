@@ -257,8 +257,8 @@ void launch_attention_mma(const State& st, int S, int layer, const bf16* q, KvVi
     // four heads per CTA when that still fills the machine, else two
     const long rows = (long)st.nb * S;
     static const int env_hpc = getenv("HBSJD_ATT_HPC") ? atoi(getenv("HBSJD_ATT_HPC")) : 0;  // tuning aid
-    if (env_hpc == 2) return launch_hpc<2>(st, S, layer, q, kv, out, s);
-    if (st.Hh % 4 == 0 && rows * (st.Hh / 4) >= 2 * 148) launch_hpc<4>(st, S, layer, q, kv, out, s);
+    // two heads per CTA (48 KB of shared memory, four CTAs per SM) measured faster than four at every shape
+    if (env_hpc == 4 && st.Hh % 4 == 0 && rows * (st.Hh / 4) >= 2 * 148) launch_hpc<4>(st, S, layer, q, kv, out, s);
     else launch_hpc<2>(st, S, layer, q, kv, out, s);
 }
 

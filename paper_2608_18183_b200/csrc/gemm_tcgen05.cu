@@ -92,6 +92,49 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// CTA-pair variants (cta_group::2): the load may signal the mbarrier of the pair's leader.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void umma_f16_pair(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(acc)
+        : "memory");
+}
+// arrives on the barrier at this shared-memory offset in BOTH CTAs of the pair once the MMAs issued so far
+// have completed
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"((unsigned short)3)
+        : "memory");
+}
+
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
     uint64_t d = 0;
@@ -104,8 +147,8 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
 }
 
 // Instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t umma_idesc(int bn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+__host__ __device__ constexpr uint32_t umma_idesc(int bn, int bm = BM) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(bm >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t acc) {
@@ -137,11 +180,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int BN>
+// PAIR: two CTAs of a cluster compute one 256 x BN tile with cta_group::2 MMAs; each CTA stages its own 128 rows
+// of A and its own BN/2 rows of W, which cuts the operand bytes per FLOP by a third against a 128 x BN tile.
+template <int BN, bool PAIR = false>
 struct Cfg {
-    static constexpr int STAGES = 4;
+    static constexpr int STAGES = PAIR ? 6 : 4;
     static constexpr int A_BYTES = BM * BK * 2;
-    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;  // two accumulators
     static constexpr int STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffers x (32 rows x 128 bytes)
@@ -155,14 +200,18 @@ struct RowDst {
     size_t kvoff; // element offset of the row's K/V vector in the page pool
 };
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_constant__ CUtensorMap map_a,
                                                               const __grid_constant__ CUtensorMap map_w,
                                                               const __grid_constant__ CUtensorMap map_c,
                                                               const GemmArgs g) {
-    using cfg = Cfg<BN>;
+    using cfg = Cfg<BN, PAIR>;
     extern __shared__ unsigned char smem_raw[];
     pdl_trigger();
+    const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader of the pair
+    const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;  // tile walker id
+    const int units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    constexpr int TM = PAIR ? 2 * BM : BM;                  // tile rows
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles = (raw + 1023u) & ~1023u;  // 1024-byte aligned tile ring
     const uint32_t staging = tiles + cfg::STAGES * cfg::STAGE_BYTES;  // 1024-byte aligned
@@ -177,7 +226,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int M = g.M, N = g.N;
     const int num_kb = g.K / BK;
-    const int tiles_n = N / BN, tiles_m = (M + BM - 1) / BM;
+    const int tiles_n = N / BN, tiles_m = (M + TM - 1) / TM;
     const int num_tiles = tiles_n * tiles_m;
 
     if (threadIdx.x == 0) {
@@ -187,20 +236,29 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(accf0 + 8 * b, 1);
-            mbar_init(acce0 + 8 * b, 4);  // one arrival per epilogue warp
+            mbar_init(acce0 + 8 * b, PAIR ? 8 : 4);  // one arrival per epilogue warp (of both CTAs)
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                         smem_u32((const void*)tmem_slot)),
-                     "r"((uint32_t)cfg::TMEM_COLS)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {  // the same warp of both CTAs allocates the same columns in both
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32((const void*)tmem_slot)),
+                         "r"((uint32_t)cfg::TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                             smem_u32((const void*)tmem_slot)),
+                         "r"((uint32_t)cfg::TMEM_COLS)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (PAIR) cluster_sync_all();  // both CTAs' barriers are initialised before either signals the other
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();  // everything above is on-chip set-up; operands of the previous kernel are read from here on
@@ -209,8 +267,9 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
             uint32_t kc = 0;
-            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x) {
-                const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+            for (int tile = unit; tile < num_tiles; tile += units) {
+                const int m0 = (tile / tiles_n) * TM + (int)rank * BM;
+                const int n0 = (tile % tiles_n) * BN + (PAIR ? (int)rank * (BN / 2) : 0);
                 bool ok = true;
                 for (int kb = 0; kb < num_kb; ++kb, ++kc) {
                     const uint32_t s = kc % cfg::STAGES, ph = (kc / cfg::STAGES) & 1u;
@@ -221,19 +280,27 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                         break;
                     }
                     const uint32_t a_dst = tiles + s * cfg::STAGE_BYTES;
-                    mbar_expect_tx(full0 + 8 * s, cfg::STAGE_BYTES);
-                    tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
-                    tma_load_2d(a_dst + cfg::A_BYTES, &map_w, kb * BK, n0, full0 + 8 * s);
+                    if (PAIR) {
+                        // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
+                        const uint32_t lead_full = map_to_rank(full0 + 8 * s, 0);
+                        if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * cfg::STAGE_BYTES);
+                        tma_load_2d_pair(a_dst, &map_a, kb * BK, m0, lead_full);
+                        tma_load_2d_pair(a_dst + cfg::A_BYTES, &map_w, kb * BK, n0, lead_full);
+                    } else {
+                        mbar_expect_tx(full0 + 8 * s, cfg::STAGE_BYTES);
+                        tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
+                        tma_load_2d(a_dst + cfg::A_BYTES, &map_w, kb * BK, n0, full0 + 8 * s);
+                    }
                 }
                 if (!ok) break;
             }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc(BN);
+        if (lane == 0 && rank == 0) {  // in a pair only the leader issues
+            constexpr uint32_t idesc = umma_idesc(BN, TM);
             uint32_t kc = 0, j = 0;
-            for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++j) {
+            for (int tile = unit; tile < num_tiles; tile += units, ++j) {
                 const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
                 bool ok = mbar_wait(acce0 + 8 * buf, aph ^ 1u, abort_flag);  // epilogue drained this accumulator
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -248,25 +315,33 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     const uint32_t a_src = tiles + s * cfg::STAGE_BYTES;
                     const uint32_t b_src = a_src + cfg::A_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k)
-                        umma_f16(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc,
-                                 (kb | k) != 0 ? 1u : 0u);
-                    umma_commit(empty0 + 8 * s);  // frees the stage once these MMAs have read it
+                    for (int k = 0; k < BK / 16; ++k) {
+                        if (PAIR)
+                            umma_f16_pair(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc,
+                                          (kb | k) != 0 ? 1u : 0u);
+                        else
+                            umma_f16(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc,
+                                     (kb | k) != 0 ? 1u : 0u);
+                    }
+                    // frees the stage (in both CTAs of a pair) once these MMAs have read it
+                    if (PAIR) umma_commit_pair(empty0 + 8 * s);
+                    else umma_commit(empty0 + 8 * s);
                 }
                 if (!ok) {
                     *abort_flag = 1;
                     atomicExch(g.error_flag, 2);
                     break;
                 }
-                umma_commit(accf0 + 8 * buf);  // accumulator complete
+                if (PAIR) umma_commit_pair(accf0 + 8 * buf);  // accumulator complete
+                else umma_commit(accf0 + 8 * buf);
             }
         }
     } else {
         // ---------------------------------------------------------------- epilogue warps 2..5
         const int quarter = warp & 3;  // TMEM lanes 32*quarter .. 32*quarter+31 belong to this warp
         uint32_t j = 0, nchunk = 0;
-        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++j) {
-            const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        for (int tile = unit; tile < num_tiles; tile += units, ++j) {
+            const int m0 = (tile / tiles_n) * TM + (int)rank * BM, n0 = (tile % tiles_n) * BN;
             const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
             if (!mbar_wait(accf0 + 8 * buf, aph, abort_flag)) {
                 if (lane == 0) {
@@ -292,6 +367,19 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 if (rd.valid) {
                     rd.s = st.slot_c[slot] + i;
                     rd.kvoff = g.kv.offset(g.layer, br * st.Bmax + st.slot_img[slot], rd.s);
+                }
+            }
+            // cos/sin of this row's sequence index, fetched once per tile (all loads in flight together):
+            // rotation pairs 0..15 and 16..31 of a head (head sizes 64: both halves; 32: the first)
+            float4 rope_lo[8], rope_hi[8];
+            if (EPI == EPI_QKV && rd.valid && n0 < 2 * g.st.D) {
+                const int half = g.st.dh / 2;
+                const float4* tab = reinterpret_cast<const float4*>(g.rope_cs + (size_t)rd.s * half * 2);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) rope_lo[v] = tab[v];
+                if (half > 16) {
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) rope_hi[v] = tab[8 + v];
                 }
             }
 #pragma unroll 1
@@ -340,7 +428,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     for (int v = 0; v < 8; ++v) {
                         const float g0 = __uint_as_float(r[4 * v]), u0 = __uint_as_float(r[4 * v + 1]);
                         const float g1 = __uint_as_float(r[4 * v + 2]), u1 = __uint_as_float(r[4 * v + 3]);
-                        o[v] = pack_bf16x2(g0 / (1.0f + expf(-g0)) * u0, g1 / (1.0f + expf(-g1)) * u1);
+                        o[v] = pack_bf16x2(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
                     }
                     dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
                     dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
@@ -350,13 +438,11 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     const int sec = col / D, cs = col % D;  // 0 q, 1 k, 2 v; a tile never straddles sections
                     uint32_t o[16];
                     if (sec < 2) {
-                        const int half = st.dh / 2;
-                        const int e0 = (cs % st.dh) / 2;  // first rotation pair of this chunk within its head
-                        const float4* tab =
-                            reinterpret_cast<const float4*>(g.rope_cs + ((size_t)rd.s * half + e0) * 2);
+                        // the chunk's 16 rotation pairs: first or second half of the row's cos/sin table
+                        const bool hi = ((cs % st.dh) / 2) >= 16;
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
-                            const float4 t = tab[v];  // cos, sin of pairs 2v and 2v+1
+                            const float4 t = hi ? rope_hi[v] : rope_lo[v];  // cos, sin of pairs 2v and 2v+1
                             const float a0 = __uint_as_float(r[4 * v]), b0 = __uint_as_float(r[4 * v + 1]);
                             const float a1 = __uint_as_float(r[4 * v + 2]), b1 = __uint_as_float(r[4 * v + 3]);
                             o[2 * v] = pack_bf16x2(a0 * t.x - b0 * t.y, a0 * t.y + b0 * t.x);
@@ -376,17 +462,26 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+            if (lane == 0) {
+                if (PAIR) mbar_arrive_cluster(map_to_rank(acce0 + 8 * buf, 0));  // the leader's MMA thread waits
+                else mbar_arrive(acce0 + 8 * buf);
+            }
         }
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if (PAIR) cluster_sync_all();  // neither CTA leaves while the other may still read its tiles or barriers
     if (warp == 1) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                     "r"((uint32_t)cfg::TMEM_COLS)
-                     : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)cfg::TMEM_COLS)
+                         : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                         "r"((uint32_t)cfg::TMEM_COLS)
+                         : "memory");
     }
 }
 
@@ -447,11 +542,26 @@ template <int BN, int EPI>
 cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
                    cudaStream_t s) {
     static int configured[64] = {0};
-    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<BN, EPI>, Cfg<BN>::SMEM, configured);
+    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<BN, EPI, false>, Cfg<BN>::SMEM, configured);
     if (e0 != cudaSuccess) return e0;
     const int tiles = (g.N / BN) * ((g.M + BM - 1) / BM);
     const int grid = tiles < num_sms() ? tiles : num_sms();
-    return launch_k(k_gemm_tcgen05<BN, EPI>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<BN>::SMEM, s, ma, mw, mc, g);
+    return launch_k(k_gemm_tcgen05<BN, EPI, false>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<BN>::SMEM, s, ma, mw,
+                    mc, g);
+}
+
+// CTA pairs: 256 x 256 tiles, one cluster of two CTAs per pair of SMs.
+template <int EPI>
+cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
+                        cudaStream_t s) {
+    static int configured[64] = {0};
+    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<256, EPI, true>, Cfg<256, true>::SMEM, configured);
+    if (e0 != cudaSuccess) return e0;
+    const int tiles = (g.N / 256) * ((g.M + 2 * BM - 1) / (2 * BM));
+    const int pairs = num_sms() / 2;
+    const int grid = 2 * (tiles < pairs ? tiles : pairs);
+    return launch_kc(k_gemm_tcgen05<256, EPI, true>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<256, true>::SMEM, s, 2,
+                     ma, mw, mc, g);
 }
 
 template <int EPI>
@@ -461,6 +571,7 @@ cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mw, cons
         case 32: return launch<32, EPI>(ma, mw, mc, g, s);
         case 64: return launch<64, EPI>(ma, mw, mc, g, s);
         case 128: return launch<128, EPI>(ma, mw, mc, g, s);
+        case 512: return launch_pair<EPI>(ma, mw, mc, g, s);  // 256 x 256 on a CTA pair
         default: return launch<256, EPI>(ma, mw, mc, g, s);
     }
 }
@@ -482,22 +593,25 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
         snprintf(err, errlen, "gemm: N=%d is not a multiple of the tile width %d", N, bn);
         return -1;
     }
+    // large problems: 256 x 256 tiles on CTA pairs (a third less operand traffic per FLOP)
+    static const bool pair_on = !(getenv("HBSJD_GEMM_PAIR") && atoi(getenv("HBSJD_GEMM_PAIR")) == 0);
+    const bool pair = pair_on && bn == 256 && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2;
     CUtensorMap ma, mw, mc;
     memset(&mc, 0, sizeof(mc));
     if ((epi == EPI_STORE || epi == EPI_ADD) && !make_map_c(&mc, g.C, M, N)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed for the output (M=%d N=%d)", M, N);
         return -3;
     }
-    if (!make_map(&ma, A, M, K, BM) || !make_map(&mw, W, N, K, bn)) {
+    if (!make_map(&ma, A, M, K, BM) || !make_map(&mw, W, N, K, pair ? 128 : bn)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
         return -3;
     }
     cudaError_t e;
     switch (epi) {
-        case EPI_STORE: e = launch_bn<EPI_STORE>(bn, ma, mw, mc, g, s); break;
-        case EPI_ADD: e = launch_bn<EPI_ADD>(bn, ma, mw, mc, g, s); break;
-        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(bn, ma, mw, mc, g, s); break;
-        default: e = launch_bn<EPI_QKV>(bn, ma, mw, mc, g, s); break;
+        case EPI_STORE: e = launch_bn<EPI_STORE>(pair ? 512 : bn, ma, mw, mc, g, s); break;
+        case EPI_ADD: e = launch_bn<EPI_ADD>(pair ? 512 : bn, ma, mw, mc, g, s); break;
+        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(pair ? 512 : bn, ma, mw, mc, g, s); break;
+        default: e = launch_bn<EPI_QKV>(pair ? 512 : bn, ma, mw, mc, g, s); break;
     }
     if (e != cudaSuccess) {
         snprintf(err, errlen, "gemm launch: %s", cudaGetErrorString(e));

@@ -26,7 +26,8 @@ def ctx_fp32():
 
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (128, 64, 128), (64, 32, 64), (200, 384, 128), (1000, 768, 768),
                                    (1024, 2304, 768), (333, 4096, 768), (1024, 768, 2048), (4096, 1024, 2816),
-                                   (2048, 16384, 1024), (1, 128, 64)])
+                                   (2048, 16384, 1024), (1, 128, 64), (8192, 3072, 1024), (8192, 1024, 1024),
+                                   (5000, 2048, 512), (4999, 5632, 1024), (2304, 16384, 256)])
 def test_bf16_gemm_matches_fp32_product(ctx_bf16, M, N, K):
     import torch
     g = torch.Generator(device="cuda").manual_seed(M * 7 + N * 3 + K)
