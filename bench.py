@@ -122,6 +122,32 @@ def run_reference(args, w, weights, toks, k, lab):
     print(json.dumps(line))
 
 
+def rank_inputs(w, rank):
+    """Each rank rolls out its own batch (replicas, no exchange step): the input seed is offset by the rank."""
+    return synth.make_inputs(w, seed=w.input_seed + 1000 * rank)
+
+
+def max_over_ranks(ms_local, dist, device):
+    """Step time of the job = the slowest rank's device time (an all-reduce MAX when there are several ranks)."""
+    if dist is None:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([float(ms_local)], device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_tokens_per_s(tokens_per_step_local, steps, dist, device, ms):
+    """Whole-job throughput: tokens committed by all ranks in the timed steps / the max-over-ranks time."""
+    total = float(tokens_per_step_local * steps)
+    if dist is not None:
+        import torch
+        t = torch.tensor([total], device=device, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.SUM)
+        total = float(t.item())
+    return total / (ms * 1e-3), total
+
+
 def workload_config(w):
     s = w.shape
     return {"workload": f"{w.name}: L{s.n_layers} D{s.dim} H{s.n_heads} F{s.ffn_hidden} V{s.vocab} "
@@ -151,7 +177,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     weights = synth.make_weights(w.shape, w.weight_seed)
-    toks, k, lab = synth.make_inputs(w, seed=w.input_seed + 1000 * rank)
+    toks, k, lab = rank_inputs(w, rank)
 
     if args.impl == "reference":
         run_reference(args, w, weights, toks, k, lab)
@@ -195,11 +221,7 @@ def main():
         stats = [fn(args.warmup + i) for i in range(steps)]
         e1.record()
         torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
         barrier()
         return ms, stats
 
@@ -241,10 +263,10 @@ def main():
                        "frac": gbs / pk["hbm_gbs"], "ms_per_step": c["ms"] / args.steps,
                        "share_of_step": c["ms"] / ms_prof if ms_prof > 0 else None}
 
-    total_tokens = tokens_per_step * args.steps * world
+    value, total_tokens = job_tokens_per_s(tokens_per_step, args.steps, dist, "cuda", ms)
     committed = sum(s["committed"] for s in stats)
     forwards = sum(s["image_forwards"] for s in stats)
-    line = {"metric": METRIC, "value": total_tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": w.shape.dtype, "data": "synthetic",
             "config": workload_config(w) | {"exec_mode": args.exec_mode, "gamma": gamma},
