@@ -29,6 +29,9 @@ from paper_2608_18183_b200 import synth  # noqa: E402
 
 METRIC = "committed image tokens/sec per B200 rollout; mean accepted tokens/forward"
 UNIT = "tokens/s"
+# DRAM bytes per GEMM launch (read + write) from the ncu capture summarised in
+# profiles/gemm_tcgen05_rollout_L.md: mean over the 97 GEMM launches of one Full round of workload L.
+NCU_GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"L": 54.9e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -164,7 +167,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="L", choices=sorted(synth.WORKLOADS))
-    ap.add_argument("--gamma-frac", type=float, default=0.5, help="Full->Compact threshold as a fraction of the batch")
+    ap.add_argument("--gamma-frac", type=float, default=1.0,
+                    help="Eq. 6 threshold as a fraction of the batch (Full iff live > threshold); 1.0 = the measured "
+                         "optimum, always Compact (profiles/exec_mode_and_window_sweep.md); 0 = always Full")
     ap.add_argument("--exec-mode", default="hybrid", choices=["full", "compact", "hybrid"])
     ap.add_argument("--window", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -248,7 +253,8 @@ def main():
     gemm_tflops = g["work"] / (g["ms"] * 1e-3) / 1e12 if g["ms"] > 0 else 0.0
     roof = {"bound": "tensor", "kernel": "k_gemm_tcgen05 (all decoder GEMMs)", "achieved": gemm_tflops,
             "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-            "frac": gemm_tflops / pk["bf16_tflops_sustained"], "traffic": None,
+            "frac": gemm_tflops / pk["bf16_tflops_sustained"],
+            "traffic": NCU_GEMM_TRAFFIC_BYTES_PER_LAUNCH.get(w.name) if not args.window else None,
             "peak_source": f"{pk['source']} sustained bf16 (kernel timed inside a long step)",
             "avg_launch_ms": g["ms"] / max(g["launches"], 1), "launches": g["launches"],
             "share_of_step": g["ms"] / ms_prof if ms_prof > 0 else None}

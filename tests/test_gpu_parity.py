@@ -1,11 +1,13 @@
 """Parity of the CUDA rollout path (through the C ABI) with the CPU oracle.
 
 Tolerances:
-  forward logits      max-abs <= 1e-4 (fp32 model); bf16 model: <= 2e-2 x max(1, std of the logits).
-                      bf16 rounding of the activations is a RELATIVE error (unit roundoff 2^-9 per
-                      rounding point), so the absolute logit error grows with the logit scale.  With a
-                      plain N(0, 0.02) head (logit std < 1) the literal bound 2e-2 holds and is asserted
-                      below; the benchmark's entropy-scaled heads have logit std 2.5-4.
+  forward logits      max-abs <= 1e-4 (fp32 model); bf16 model: <= max(2e-2, 5.5 s) with
+                      s = std(logits) (2^-9 / sqrt 3) sqrt(6 L + 1) (gpu_util.bf16_logit_tol): bf16 rounding
+                      of the activations is a RELATIVE error per rounding point that accumulates over the
+                      layers, so the absolute logit error grows with the logit scale and the depth; the mean
+                      absolute error must stay below s.  With a plain N(0, 0.02) head (logit std < 1) the
+                      literal bound 2e-2 holds and is asserted below; the benchmark's entropy-scaled heads
+                      have logit std 2.5-4.5.
   probabilities       |p_gpu - p_oracle(gpu logits)| <= 1e-6 + 1e-4 p   (expf vs exp, fp32 sums)
   verify/commit/refresh, initial windows, compaction tables: bit-exact given the same p, q, words
   end to end (lockstep): plain head: >= 99 % of committed tokens identical and every differing decision
@@ -84,7 +86,8 @@ def test_tiny_bf16_cfg_topk_lockstep(greedy):
     model = O.Model(w.shape, G.weights_for(w))
     ctx = _ctx(w)
     rep = G.lockstep(ctx, model, w, toks, k, lab, 11, greedy=greedy)
-    tol = 2e-2 * max(1.0, rep["logit_std"])
+    std, tol = G.bf16_logit_tol(rep["logit_std"], w.shape.n_layers)
+    assert rep["abs_err_sum"] / rep["abs_err_n"] <= std
     _check_report(rep, tol, min_same=0.95, margin=float(np.expm1(2 * tol)))
     ctx.hbsjd_destroy()
 
@@ -115,7 +118,8 @@ def test_small_bf16_wide_windows_multi_page(W):
     model = O.Model(w.shape, G.weights_for(w))
     ctx = _ctx(w)
     rep = G.lockstep(ctx, model, w, toks, k, lab, 21, max_rounds=6)
-    tol = 2e-2 * max(1.0, rep["logit_std"])
+    std, tol = G.bf16_logit_tol(rep["logit_std"], w.shape.n_layers)
+    assert rep["abs_err_sum"] / rep["abs_err_n"] <= std
     _check_report(rep, tol, min_same=0.93, margin=float(np.expm1(2 * tol)))
     ctx.hbsjd_destroy()
 
