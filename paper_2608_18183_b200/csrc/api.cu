@@ -132,11 +132,12 @@ KvView kv_view(const hbsjd_ctx* c) {
     return kv;
 }
 
+// m_cap: row capacity of the A and C buffers when they are the context's own (0: exactly M rows)
 template <typename TA>
-int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate);
+int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int m_cap = 0);
 
 template <>
-int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
+int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int) {
     const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
     launch_gemm_simt<float>((const float*)A, (const float*)W, C, M, N, K, accumulate, c->stream);
     prof_end(c, ps);
@@ -145,10 +146,11 @@ int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int
 }
 
 template <>
-int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
+int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
+               int m_cap) {
     c->launches++;
     const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
-    const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, 0,
+    const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, 0, m_cap,
                                     c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err));
     prof_end(c, ps);
     return rc == 0 ? 0 : (rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA);
@@ -159,6 +161,7 @@ template <typename TA>
 int forward(hbsjd_ctx* c, int S, bool want_logits) {
     const State& st = c->st;
     const int M = st.nb * S * st.W, D = st.D, F = st.F;
+    const int Mcap = 2 * c->Bmax * c->Wmax;  // row capacity of the activation buffers
     cudaStream_t s = c->stream;
     const KvView kv = kv_view(c);
     launch_embed<TA>(st, S, (const TA*)c->tok_emb, (const TA*)c->cls_emb, c->h, s);
@@ -177,7 +180,7 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
             // QKV projection with RoPE and the paged KV write in its epilogue
             const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D);
             rc = gemm_tcgen05_qkv((const bf16*)c->a, (const bf16*)w.w_qkv, (bf16*)c->q, st, S, l, c->rope_cs, kv,
-                                  c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
+                                  Mcap, c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
             prof_end(c, ps);
             if (rc) return rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
             c->launches += 2;
@@ -199,13 +202,13 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
             prof_end(c, ps);
             c->launches++;
         }
-        if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1))) return rc;
+        if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1, Mcap))) return rc;
         norm(c->h, w.g_ffn);
         c->launches++;
         if constexpr (std::is_same<TA, bf16>::value) {
             // gate/up projection with SwiGLU in its epilogue (gate and up rows interleaved at load time)
             const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D);
-            rc = gemm_tcgen05_swiglu((const bf16*)c->a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D,
+            rc = gemm_tcgen05_swiglu((const bf16*)c->a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D, Mcap,
                                      c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
             prof_end(c, ps);
             if (rc) return rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
@@ -215,13 +218,13 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
             launch_swiglu<TA>(c->gu, (TA*)c->act, M, F, s);
             c->launches++;
         }
-        if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1))) return rc;
+        if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1, Mcap))) return rc;
     }
     if (want_logits) {
         norm(c->h, c->g_out);
         c->launches++;
         int rc;
-        if ((rc = gemm<TA>(c, c->a, c->w_head, c->logits, M, st.V, D, 0))) return rc;
+        if ((rc = gemm<TA>(c, c->a, c->w_head, c->logits, M, st.V, D, 0, Mcap))) return rc;
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {

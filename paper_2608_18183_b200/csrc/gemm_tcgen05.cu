@@ -21,6 +21,9 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <functional>
+#include <mutex>
+#include <unordered_map>
 
 #include "internal.h"
 
@@ -184,7 +187,9 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 // of A and its own BN/2 rows of W, which cuts the operand bytes per FLOP by a third against a 128 x BN tile.
 template <int BN, bool PAIR = false>
 struct Cfg {
-    static constexpr int STAGES = PAIR ? 6 : 4;
+    // as many stages as fit beside the 32 KB epilogue staging: small tiles are latency-bound (one TMA round
+    // trip per ring revolution), so a narrow tile gets a deep ring
+    static constexpr int STAGES = PAIR ? 6 : (BN >= 256 ? 4 : (BN == 128 ? 6 : (BN == 64 ? 8 : 9)));
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -240,6 +245,11 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0 && lane == 0) {  // descriptor fetch off the critical path
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
+        if (EPI == EPI_STORE || EPI == EPI_ADD) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
     }
     if (warp == 1) {
         if (PAIR) {  // the same warp of both CTAs allocates the same columns in both
@@ -503,8 +513,42 @@ EncodeFn get_encode() {
     return fn;
 }
 
+// Encoded tensor maps are cached by (address, extents, box, type): encoding costs microseconds on the host,
+// and a round issues hundreds of GEMMs over the same few buffers.
+struct MapKey {
+    const void* base;
+    int rows, inner, box_rows, kind;
+    bool operator==(const MapKey& o) const {
+        return base == o.base && rows == o.rows && inner == o.inner && box_rows == o.box_rows && kind == o.kind;
+    }
+};
+struct MapKeyHash {
+    size_t operator()(const MapKey& k) const {
+        size_t h = std::hash<const void*>()(k.base);
+        h = h * 1000003u ^ (size_t)k.rows;
+        h = h * 1000003u ^ (size_t)k.inner;
+        h = h * 1000003u ^ (size_t)(k.box_rows * 4 + k.kind);
+        return h;
+    }
+};
+std::mutex g_map_mu;
+std::unordered_map<MapKey, CUtensorMap, MapKeyHash> g_map_cache;
+
+bool cached_map(CUtensorMap* out, const MapKey& key, bool (*encode)(CUtensorMap*, const void*, int, int, int)) {
+    std::lock_guard<std::mutex> lock(g_map_mu);
+    auto it = g_map_cache.find(key);
+    if (it != g_map_cache.end()) {
+        *out = it->second;
+        return true;
+    }
+    if (g_map_cache.size() > 4096) g_map_cache.clear();
+    if (!encode(out, key.base, key.rows, key.inner, key.box_rows)) return false;
+    g_map_cache.emplace(key, *out);
+    return true;
+}
+
 // 2D bf16 row-major [rows, K] tensor, box = [box_rows, 64], 128-byte swizzle, zero fill out of bounds.
-bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+bool encode_map_ab(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
     EncodeFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
@@ -527,17 +571,25 @@ int num_sms() {
     return n;
 }
 
+bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+    return cached_map(map, MapKey{base, rows, K, box_rows, 0}, encode_map_ab);
+}
+
 // fp32 row-major [rows, N] output, box = 32 columns (128 bytes) x 32 rows, 128-byte swizzle.
-bool make_map_c(CUtensorMap* map, const float* base, int rows, int N) {
+bool encode_map_c(CUtensorMap* map, const void* base, int rows, int N, int) {
     EncodeFn enc = get_encode();
     if (!enc) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)N * 4};
     const cuuint32_t box[2] = {32, 32};
     const cuuint32_t estr[2] = {1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool make_map_c(CUtensorMap* map, const float* base, int rows, int N) {
+    return cached_map(map, MapKey{base, rows, N, 32, 1}, encode_map_c);
 }
 
 template <int BN, int EPI>
@@ -578,8 +630,11 @@ cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mw, cons
     }
 }
 
-int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int max_bn, cudaStream_t s, char* err,
-        size_t errlen) {
+// m_cap >= M: row extent given to the A and C tensor maps (the capacity of the caller's buffers), so that one
+// cached map serves every M; rows between M and m_cap are padding (read as they are, never stored past M's
+// last 32-row block).  0: use M.
+int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int max_bn, int m_cap, cudaStream_t s,
+        char* err, size_t errlen) {
     const int M = g.M, N = g.N, K = g.K;
     if (M <= 0) return 0;
     if (K % BK != 0 || N % 32 != 0 || (((uintptr_t)A | (uintptr_t)W) & 15)) {
@@ -600,11 +655,12 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
     const bool pair = pair_on && bn == 256 && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2;
     CUtensorMap ma, mw, mc;
     memset(&mc, 0, sizeof(mc));
-    if ((epi == EPI_STORE || epi == EPI_ADD) && !make_map_c(&mc, g.C, M, N)) {
+    const int map_rows = m_cap >= M ? m_cap : M;
+    if ((epi == EPI_STORE || epi == EPI_ADD) && !make_map_c(&mc, g.C, map_rows, N)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed for the output (M=%d N=%d)", M, N);
         return -3;
     }
-    if (!make_map(&ma, A, M, K, BM) || !make_map(&mw, W, N, K, pair ? 128 : bn)) {
+    if (!make_map(&ma, A, map_rows, K, BM) || !make_map(&mw, W, N, K, pair ? 128 : bn)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
         return -3;
     }
@@ -636,7 +692,7 @@ int gemm_tcgen05_tile_n(int M, int N) {
 }
 
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
-                     int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+                     int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
     if ((uintptr_t)C & 15) {
         snprintf(err, errlen, "gemm: C must be 16-byte aligned");
         return -1;
@@ -647,10 +703,10 @@ int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K
     g.N = N;
     g.K = K;
     g.error_flag = error_flag;
-    return run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, s, err, errlen);
+    return run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, m_cap, s, err, errlen);
 }
 
-int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K,
+int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
                         int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
     GemmArgs g{};
     g.out = act;
@@ -658,12 +714,12 @@ int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, i
     g.N = F2;
     g.K = K;
     g.error_flag = error_flag;
-    return run(EPI_SWIGLU, A, W13_interleaved, g, 0, 256, s, err, errlen);
+    return run(EPI_SWIGLU, A, W13_interleaved, g, 0, 256, m_cap, s, err, errlen);
 }
 
 int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, int S, int layer,
-                     const float* rope_cs, const KvView& kv, int32_t* error_flag, cudaStream_t s, char* err,
-                     size_t errlen) {
+                     const float* rope_cs, const KvView& kv, int m_cap, int32_t* error_flag, cudaStream_t s,
+                     char* err, size_t errlen) {
     GemmArgs g{};
     g.out = q;
     g.M = st.nb * S * st.W;
@@ -678,7 +734,7 @@ int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, 
     // a tile must lie inside one of the q / k / v sections and start on a rotation-pair boundary
     int max_bn = 256;
     while (st.D % max_bn != 0) max_bn >>= 1;
-    return run(EPI_QKV, A, Wqkv, g, 0, max_bn, s, err, errlen);
+    return run(EPI_QKV, A, Wqkv, g, 0, max_bn, m_cap, s, err, errlen);
 }
 
 }  // namespace hbsjd

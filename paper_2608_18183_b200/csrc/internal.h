@@ -103,16 +103,17 @@ void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_s
 // C[M,N] fp32 (+)= A[M,K] bf16 . W[N,K]^T bf16.  force_bn: 0 = choose the tile width from the shape.
 // error_flag: device int set non-zero if a bounded pipeline wait gave up.  Returns 0, or a negative
 // code with a message in err.
+// m_cap (>= M, or 0): row capacity of the A and C buffers; lets one cached tensor map serve every M.
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
-                     int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
+                     int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
 int gemm_tcgen05_tile_n(int M, int N);
 // act[M, F] bf16 = silu(gate) * up, from A[M,K] . W13i^T where W13i[2F, K] holds gate row f at 2f, up row f at 2f+1.
-int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K,
+int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
                         int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
 // QKV projection of the normed activations A[M, D] with the 2D RoPE and the paged KV write fused:
 // q[M, D] bf16 rotated; rotated k and v stored at each row's (cache row, sequence index).
 int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, int S, int layer,
-                     const float* rope_cs, const KvView& kv, int32_t* error_flag, cudaStream_t s, char* err,
-                     size_t errlen);
+                     const float* rope_cs, const KvView& kv, int m_cap, int32_t* error_flag, cudaStream_t s,
+                     char* err, size_t errlen);
 
 }  // namespace hbsjd
