@@ -20,6 +20,7 @@
 
 #include <cstdio>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <functional>
 #include <mutex>
@@ -479,7 +480,9 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 else mbar_arrive(acce0 + 8 * buf);
             }
         }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        // the staging tiles must have been read before shared memory is released; the global writes
+        // themselves complete like any other store before dependent kernels pass their grid dependency
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
     }
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -644,7 +647,7 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
     }
     static const int env_bn = getenv("HBSJD_GEMM_BN") ? atoi(getenv("HBSJD_GEMM_BN")) : 0;  // tuning aid
     if (!force_bn && env_bn && N % env_bn == 0) force_bn = env_bn;
-    int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N);
+    int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N, K);
     while (bn > max_bn) bn >>= 1;
     if (bn < 32 || N % bn != 0) {
         snprintf(err, errlen, "gemm: N=%d is not a multiple of the tile width %d", N, bn);
@@ -680,15 +683,29 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
 
 }  // namespace
 
-// Widest tile that still gives every SM a tile; small problems take narrower tiles.
-int gemm_tcgen05_tile_n(int M, int N) {
+// Tile width by a small cost model: waves of tiles over the SMs times the time of one tile, where a tile costs
+// a fixed part plus, per 64-wide k-block, the larger of the TMA round trip amortised over the ring and the MMA
+// time of a 128 x BN x 64 block.  Large problems end up with 256 (CTA pairs), small ones with the widest tile
+// that still fits one wave.
+int gemm_tcgen05_tile_n(int M, int N, int K) {
     const long tiles_m = (M + BM - 1) / BM;
-    const int sms = 148;
-    for (int bn = 256; bn >= 64; bn >>= 1)
-        if (N % bn == 0 && tiles_m * (N / bn) >= sms) return bn;
-    for (int bn = 32; bn <= 256; bn <<= 1)
-        if (N % bn == 0) return bn;
-    return 32;
+    const int sms = 148, num_kb = K / BK;
+    // enough 256-wide tiles for every SM: the wide tile has the lowest operand traffic per FLOP
+    if (N % 256 == 0 && tiles_m * (N / 256) >= sms) return 256;
+    int best = 0;
+    float best_cost = 0.f;
+    for (int bn = 256; bn >= 32; bn >>= 1) {
+        if (N % bn != 0) continue;
+        const long tiles = tiles_m * (N / bn);
+        const long waves = (tiles + sms - 1) / sms;
+        const float per_kb = fmaxf(0.12f, 0.51f * (float)bn / 256.0f);  // microseconds
+        const float cost = (float)waves * (1.0f + (float)num_kb * per_kb);
+        if (best == 0 || cost < best_cost * 0.98f) {  // prefer the wider tile on a tie
+            best = bn;
+            best_cost = cost;
+        }
+    }
+    return best ? best : 32;
 }
 
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,

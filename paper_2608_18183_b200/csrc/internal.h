@@ -106,7 +106,7 @@ void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_s
 // m_cap (>= M, or 0): row capacity of the A and C buffers; lets one cached tensor map serve every M.
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
                      int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
-int gemm_tcgen05_tile_n(int M, int N);
+int gemm_tcgen05_tile_n(int M, int N, int K);
 // act[M, F] bf16 = silu(gate) * up, from A[M,K] . W13i^T where W13i[2F, K] holds gate row f at 2f, up row f at 2f+1.
 int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
                         int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
