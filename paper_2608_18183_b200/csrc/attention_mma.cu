@@ -79,22 +79,41 @@ __global__ void __launch_bounds__(QB * HPC * 32) k_attention_mma(State st, int S
     const int total_keys = c + n;
     const int nblocks = (total_keys + KB - 1) / KB;
 
-    // ---- K/V block loader: all threads, 16-byte chunks; keys >= total_keys are zero-filled
+    // ---- K/V block loader: all threads, 16-byte chunks; keys >= total_keys are zero-filled.
+    // The row's page-table entries are fetched once (not once per block on the critical path of the copies),
+    // and each thread's chunk coordinates are fixed for the whole kernel.
+    __shared__ int s_pages[32];
+    if (tid < 32 && tid < kv.pages_per_row && tid * kv.page < total_keys) s_pages[tid] = kv.table[crow * kv.pages_per_row + tid];
+    __syncthreads();
+    constexpr int CHUNKS = HPC * 2 * KB * 8;       // 16-byte chunks per block
+    constexpr int PER_THREAD = (CHUNKS + NT - 1) / NT;  // chunks each thread copies per block
+    uint32_t c_dst[PER_THREAD];                     // shared-memory offset inside a stage
+    int c_src[PER_THREAD];                          // element offset from the block's first key row, K or V pool
+    int c_row[PER_THREAD];
+#pragma unroll
+    for (int u = 0; u < PER_THREAD; ++u) {
+        const int idx = tid + u * NT;
+        const int chunk = idx & 7;
+        const int row = (idx >> 3) & (KB - 1);
+        const int kvsel = (idx >> 8) & 1;  // 0 = K, 1 = V   (8 chunks * 32 rows = 256)
+        const int hh = idx >> 9;
+        c_dst[u] = hh * HEAD_STAGE + kvsel * (KB * DH * 2) + tile_off(row, chunk);
+        c_src[u] = row * D + (head0 + hh) * DH + chunk * 8;
+        c_row[u] = idx < CHUNKS ? (row | (kvsel << 16)) : -1;
+    }
+    const size_t layer_base = (size_t)layer * kv.n_pages * kv.page * (size_t)D;
     auto load_block = [&](int blk, int stage) {
         const int key0 = blk * KB;
         // one page holds whole blocks (page size is a multiple of 32)
-        const size_t base = kv.offset(layer, crow, key0);
-        const bf16* kb = (const bf16*)kv.k + base + head0 * DH;
-        const bf16* vb = (const bf16*)kv.v + base + head0 * DH;
+        const size_t base = layer_base + ((size_t)s_pages[key0 / kv.page] * kv.page + (key0 % kv.page)) * (size_t)D;
+        const bf16* kb = (const bf16*)kv.k + base;
+        const bf16* vb = (const bf16*)kv.v + base;
         const uint32_t sbase = smem_base + stage * STAGE_BYTES;
-        for (int idx = tid; idx < HPC * 2 * KB * 8; idx += NT) {
-            const int chunk = idx & 7;
-            const int row = (idx >> 3) & (KB - 1);
-            const int kvsel = (idx >> 8) & 1;  // 0 = K, 1 = V   (8 chunks * 32 rows = 256)
-            const int hh = idx >> 9;
-            const bf16* src = (kvsel ? vb : kb) + (size_t)row * D + hh * DH + chunk * 8;
-            const uint32_t dst = sbase + hh * HEAD_STAGE + kvsel * (KB * DH * 2) + tile_off(row, chunk);
-            cp_async16(dst, src, key0 + row < total_keys);
+#pragma unroll
+        for (int u = 0; u < PER_THREAD; ++u) {
+            if (c_row[u] < 0) continue;
+            const bf16* src = ((c_row[u] >> 16) ? vb : kb) + c_src[u];
+            cp_async16(sbase + c_dst[u], src, key0 + (c_row[u] & 0xffff) < total_keys);
         }
     };
 
@@ -156,17 +175,31 @@ __global__ void __launch_bounds__(QB * HPC * 32) k_attention_mma(State st, int S
                 mma_bf16(sc[nt], qa[half * 2 + 1], b2, b3);
             }
         }
-        // causal mask + online softmax (rows r0 = lane/4 and r0+8; columns (lane%4)*2 + {0,1} per n-tile)
+        // causal mask + online softmax (rows r0 = lane/4 and r0+8; columns (lane%4)*2 + {0,1} per n-tile).
+        // A block wholly at or before the warp's first query (key0 + 31 <= c + 16 wq) needs no mask; scaling
+        // a visible score is the same multiplication either way, so the two paths agree bit for bit.
         float mx0 = m0, mx1 = m1;
+        if (key0 + KB - 1 <= c + wq * 16) {
 #pragma unroll
-        for (int nt = 0; nt < 4; ++nt) {
-            const int key = key0 + nt * 8 + (lane & 3) * 2;
-            sc[nt][0] = key <= s0 ? sc[nt][0] * sl2 : -INFINITY;
-            sc[nt][1] = key + 1 <= s0 ? sc[nt][1] * sl2 : -INFINITY;
-            sc[nt][2] = key <= s1 ? sc[nt][2] * sl2 : -INFINITY;
-            sc[nt][3] = key + 1 <= s1 ? sc[nt][3] * sl2 : -INFINITY;
-            mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
-            mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+            for (int nt = 0; nt < 4; ++nt) {
+                sc[nt][0] *= sl2;
+                sc[nt][1] *= sl2;
+                sc[nt][2] *= sl2;
+                sc[nt][3] *= sl2;
+                mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+            }
+        } else {
+#pragma unroll
+            for (int nt = 0; nt < 4; ++nt) {
+                const int key = key0 + nt * 8 + (lane & 3) * 2;
+                sc[nt][0] = key <= s0 ? sc[nt][0] * sl2 : -INFINITY;
+                sc[nt][1] = key + 1 <= s0 ? sc[nt][1] * sl2 : -INFINITY;
+                sc[nt][2] = key <= s1 ? sc[nt][2] * sl2 : -INFINITY;
+                sc[nt][3] = key + 1 <= s1 ? sc[nt][3] * sl2 : -INFINITY;
+                mx0 = fmaxf(mx0, fmaxf(sc[nt][0], sc[nt][1]));
+                mx1 = fmaxf(mx1, fmaxf(sc[nt][2], sc[nt][3]));
+            }
         }
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
@@ -258,6 +291,7 @@ void launch_attention_mma(const State& st, int S, int layer, const bf16* q, KvVi
     const long rows = (long)st.nb * S;
     static const int env_hpc = getenv("HBSJD_ATT_HPC") ? atoi(getenv("HBSJD_ATT_HPC")) : 0;  // tuning aid
     // two heads per CTA (48 KB of shared memory, four CTAs per SM) measured faster than four at every shape
+    if (env_hpc == 1) return launch_hpc<1>(st, S, layer, q, kv, out, s);
     if (env_hpc == 4 && st.Hh % 4 == 0 && rows * (st.Hh / 4) >= 2 * 148) launch_hpc<4>(st, S, layer, q, kv, out, s);
     else launch_hpc<2>(st, S, layer, q, kv, out, s);
 }
