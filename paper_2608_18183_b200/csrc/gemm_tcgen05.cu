@@ -43,6 +43,7 @@ struct GemmArgs {
     bf16* out;       // SWIGLU: [M, N/2];  QKV: q [M, D]
     int M, N, K;
     int32_t* error_flag;
+    unsigned long long* timeline;  // tuning aid: when set, CTA 0 records %globaltimer stamps of its phases
     // QKV epilogue
     State st;
     int S, layer;
@@ -214,6 +215,8 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     using cfg = Cfg<BN, PAIR>;
     extern __shared__ unsigned char smem_raw[];
     pdl_trigger();
+    unsigned long long* tl = (g.timeline && blockIdx.x == 0) ? g.timeline : nullptr;
+    if (tl && threadIdx.x == 0) tl[0] = globaltimer_ns();  // kernel entry
     const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader of the pair
     const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;  // tile walker id
     const int units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -272,7 +275,9 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     if (PAIR) cluster_sync_all();  // both CTAs' barriers are initialised before either signals the other
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
+    if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns();  // set-up done
     pdl_wait();  // everything above is on-chip set-up; operands of the previous kernel are read from here on
+    if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();  // grid dependency released
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -322,6 +327,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                         ok = false;
                         break;
                     }
+                    if (tl && kc == 0) tl[3] = globaltimer_ns();  // first operands landed
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_src = tiles + s * cfg::STAGE_BYTES;
                     const uint32_t b_src = a_src + cfg::A_BYTES;
@@ -345,6 +351,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 }
                 if (PAIR) umma_commit_pair(accf0 + 8 * buf);  // accumulator complete
                 else umma_commit(accf0 + 8 * buf);
+                if (tl && j == 0) tl[4] = globaltimer_ns();  // first tile's MMAs issued
             }
         }
     } else {
@@ -362,6 +369,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (tl && j == 0 && warp == 2 && lane == 0) tl[5] = globaltimer_ns();  // first accumulator ready
             const int row = m0 + quarter * 32 + lane;
             const uint32_t tbase = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
 
@@ -482,12 +490,15 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         }
         // the staging tiles must have been read before shared memory is released; the global writes
         // themselves complete like any other store before dependent kernels pass their grid dependency
+        if (tl && warp == 2 && lane == 0) tl[6] = globaltimer_ns();  // last epilogue chunk issued
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        if (tl && warp == 2 && lane == 0) tl[7] = globaltimer_ns();  // staging drained
     }
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (PAIR) cluster_sync_all();  // neither CTA leaves while the other may still read its tiles or barriers
+    if (tl && threadIdx.x == 0) tl[8] = globaltimer_ns();  // all roles done
     if (warp == 1) {
         if (PAIR)
             asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
@@ -683,10 +694,11 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
 
 }  // namespace
 
-// Tile width by a small cost model: waves of tiles over the SMs times the time of one tile, where a tile costs
-// a fixed part plus, per 64-wide k-block, the larger of the TMA round trip amortised over the ring and the MMA
-// time of a 128 x BN x 64 block.  Large problems end up with 256 (CTA pairs), small ones with the widest tile
-// that still fits one wave.
+// Tile width by a small cost model: waves of tiles over the SMs times the time of one tile.  Measured with the
+// phase stamps of this kernel (HBSJD_GEMM_TIMELINE): a k-block of four dependent MMAs into one accumulator
+// takes about 0.285 us however narrow the tile is (the accumulation chain is latency-bound below N = 128..256)
+// and 0.51 us at N = 256; the epilogue adds about 0.15 us per 32 columns.  Large problems end up with 256
+// (CTA pairs), small ones with the widest tile that still fits one wave.
 int gemm_tcgen05_tile_n(int M, int N, int K) {
     const long tiles_m = (M + BM - 1) / BM;
     const int sms = 148, num_kb = K / BK;
@@ -698,8 +710,8 @@ int gemm_tcgen05_tile_n(int M, int N, int K) {
         if (N % bn != 0) continue;
         const long tiles = tiles_m * (N / bn);
         const long waves = (tiles + sms - 1) / sms;
-        const float per_kb = fmaxf(0.12f, 0.51f * (float)bn / 256.0f);  // microseconds
-        const float cost = (float)waves * (1.0f + (float)num_kb * per_kb);
+        const float per_kb = fmaxf(0.285f, 0.51f * (float)bn / 256.0f);  // microseconds
+        const float cost = (float)waves * (1.0f + 0.15f * (float)(bn / 32) + (float)num_kb * per_kb);
         if (best == 0 || cost < best_cost * 0.98f) {  // prefer the wider tile on a tie
             best = bn;
             best_cost = cost;
@@ -720,6 +732,22 @@ int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K
     g.N = N;
     g.K = K;
     g.error_flag = error_flag;
+    static unsigned long long* tl_dev = nullptr;
+    static const bool tl_on = getenv("HBSJD_GEMM_TIMELINE") != nullptr;
+    if (tl_on) {  // tuning aid: print the phase stamps of CTA 0 of this launch
+        if (!tl_dev) cudaMalloc((void**)&tl_dev, 16 * sizeof(unsigned long long));
+        cudaMemsetAsync(tl_dev, 0, 16 * sizeof(unsigned long long), s);
+        g.timeline = tl_dev;
+        const int rc = run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, m_cap, s, err, errlen);
+        unsigned long long h[16];
+        cudaMemcpyAsync(h, tl_dev, sizeof(h), cudaMemcpyDeviceToHost, s);
+        cudaStreamSynchronize(s);
+        fprintf(stderr, "gemm M%d N%d K%d acc%d timeline(ns): setup %llu wait %llu first_load %llu mma_issued %llu "
+                        "acc_ready %llu epi_issued %llu drained %llu done %llu\n",
+                M, N, K, accumulate, h[1] - h[0], h[2] - h[0], h[3] - h[0], h[4] - h[0], h[5] - h[0], h[6] - h[0],
+                h[7] - h[0], h[8] - h[0]);
+        return rc;
+    }
     return run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, m_cap, s, err, errlen);
 }
 
