@@ -177,6 +177,7 @@ def main():
                          "optimum, always Compact (profiles/exec_mode_and_window_sweep.md); 0 = always Full")
     ap.add_argument("--exec-mode", default="hybrid", choices=["full", "compact", "hybrid"])
     ap.add_argument("--window", type=int, default=0)
+    ap.add_argument("--verify", default="prob", choices=["prob", "greedy"], help="Eq. 5 (default) or Eq. 4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
 
@@ -209,7 +210,8 @@ def main():
 
     def params(seed):
         return binding.make_params(w.window, w.history_offset, w.cfg_scale, w.temperature, w.top_k,
-                                   binding.VERIFY_PROB, mode, gamma, seed, -1)
+                                   binding.VERIFY_GREEDY if args.verify == "greedy" else binding.VERIFY_PROB, mode,
+                                   gamma, seed, -1)
 
     d_toks, d_k, d_lab = (torch.from_numpy(x).cuda() for x in (toks, k, lab))
     d_out = torch.empty((w.batch, w.shape.T), dtype=torch.int32, device="cuda")
@@ -280,7 +282,8 @@ def main():
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": w.shape.dtype, "data": "synthetic",
-            "config": workload_config(w) | {"exec_mode": args.exec_mode, "gamma": gamma},
+            "config": workload_config(w) | {"exec_mode": args.exec_mode, "gamma": gamma,
+                                            "verify": "greedy" if args.verify == "greedy" else "probabilistic"},
             "mean_accepted_tokens_per_forward": committed / max(forwards, 1),
             "rounds_per_step": sum(s["rounds"] for s in stats) / args.steps,
             "reject_rate": sum(s["rejects"] for s in stats) / max(forwards, 1),

@@ -123,6 +123,17 @@ int hbsjd_rollout(hbsjd_ctx *c, int batch, const int32_t *prefix_tokens, const i
 int hbsjd_rollout_host(hbsjd_ctx *c, int batch, const int32_t *prefix_tokens, const int32_t *prefix_len,
                        const int32_t *class_labels, const hbsjd_params *p, int32_t *out_tokens, hbsjd_stats *stats);
 
+/* Threshold calibration of Sec. 4.3 ("a lightweight, data-independent latency test with a few verifier
+ * forwards"): times the verifier forward of a `batch`-image rollout (window, guidance on/off) with A live
+ * images, once in Full form (all `batch` slots) and once in Compact form (A slots), for
+ * A = batch, 3/4, 1/2, 1/4 and 1/8 of the batch, on a synthetic state (cursors at T/2).  *gamma_out (HOST) =
+ * the largest tested A at which Compact is not slower than Full beyond 1 % timing noise (Eq. 6 keeps Full for
+ * A > gamma); 0 if Compact
+ * is slower everywhere.  ms_full / ms_compact: HOST float[5] or NULL, the measured milliseconds in that order.
+ * Discards the context's rollout state.  Errors: HBSJD_EINVAL, HBSJD_ECUDA, HBSJD_ETIMEOUT. */
+int hbsjd_calibrate_gamma(hbsjd_ctx *c, int batch, int window, int guidance, int *gamma_out, float *ms_full,
+                          float *ms_compact);
+
 /* One verification round (Sec. 4.2 "Batched verification" .. "Independent progress") on the state left
  * by hbsjd_rollout or a previous hbsjd_round.  *live_out (HOST) = images still incomplete afterwards.
  * A sequence of hbsjd_rollout(max_rounds = 0) and hbsjd_round calls yields the same tokens as one

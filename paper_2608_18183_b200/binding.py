@@ -16,7 +16,7 @@ VERIFY_PROB, VERIFY_GREEDY = 0, 1
 EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
-EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
+EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
            "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_strerror", "hbsjd_last_error"]
 
 
@@ -83,6 +83,8 @@ def load():
         L.hbsjd_probs.argtypes = [vp, vp, vp, C.c_int, C.c_float, C.c_float, C.c_int, vp]
         L.hbsjd_verify.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
         L.hbsjd_verify_static.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
+        L.hbsjd_calibrate_gamma.argtypes = [vp, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_int),
+                                            C.POINTER(C.c_float), C.POINTER(C.c_float)]
         L.hbsjd_round.argtypes = [vp, C.POINTER(C.c_int)]
         L.hbsjd_tokens.argtypes = [vp, vp]
         L.hbsjd_destroy.argtypes = [vp]
@@ -198,6 +200,15 @@ class Context:
         self._check(self.lib.hbsjd_verify(self.h, C.byref(desc), logits.data_ptr(), q_prev.data_ptr(),
                                           p_out.data_ptr(), cursor.data_ptr(), seq.data_ptr(), delta.data_ptr(),
                                           qbase.data_ptr(), m_out.data_ptr()), "hbsjd_verify")
+
+    def hbsjd_calibrate_gamma(self, batch, window, guidance):
+        """Returns (gamma, ms_full[5], ms_compact[5]) for live = batch, 3/4, 1/2, 1/4, 1/8 of the batch."""
+        g = C.c_int(0)
+        mf, mc = (C.c_float * 5)(), (C.c_float * 5)()
+        self._check(self.lib.hbsjd_calibrate_gamma(self.h, batch, window, 1 if guidance else 0, C.byref(g), mf, mc),
+                    "hbsjd_calibrate_gamma")
+        self.batch = 0
+        return g.value, list(mf), list(mc)
 
     def hbsjd_round(self) -> int:
         live = C.c_int(0)

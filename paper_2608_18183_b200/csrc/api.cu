@@ -721,6 +721,58 @@ int hbsjd_profile_read(hbsjd_ctx* c, hbsjd_kernel_profile* out) {
     return HBSJD_OK;
 }
 
+int hbsjd_calibrate_gamma(hbsjd_ctx* c, int batch, int window, int guidance, int* gamma_out, float* ms_full,
+                          float* ms_compact) {
+    if (!c) return HBSJD_EINVAL;
+    if (!gamma_out || batch < 1 || batch > c->Bmax || window < 1 || window > c->Wmax) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_calibrate_gamma: argument out of range");
+        return HBSJD_EINVAL;
+    }
+    c->have_rollout = false;
+    State& st = c->st;
+    st.B = batch;
+    st.T = c->T;
+    st.V = c->d.vocab;
+    st.D = c->d.dim;
+    st.Hh = c->d.n_heads;
+    st.dh = c->dh;
+    st.F = c->d.ffn_hidden;
+    st.L = c->d.n_layers;
+    st.C = c->d.n_classes;
+    st.Bmax = c->Bmax;
+    st.Wmax = c->Wmax;
+    st.W = window;
+    st.H = 1;
+    st.nb = guidance ? 2 : 1;
+    const int points[5] = {batch, (3 * batch) / 4, batch / 2, batch / 4, batch / 8};
+    int gamma = 0;
+    for (int p = 0; p < 5; ++p) {
+        const int live = points[p] < 1 ? 1 : points[p];
+        float best[2] = {0.f, 0.f};
+        for (int compact = 0; compact < 2; ++compact) {
+            const int S = compact ? live : batch;
+            for (int rep = 0; rep < 4; ++rep) {  // the first repetition warms up
+                launch_calib_state(st, live, c->stream);
+                launch_setup(st, 0, compact, c->stream);
+                CK(cudaEventRecord(c->ev0, c->stream));
+                const int rc = forward_any(c, S, true);
+                if (rc) return rc;
+                CK(cudaEventRecord(c->ev1, c->stream));
+                const int rs = sync_counters(c);
+                if (rs) return rs;
+                float ms = 0.f;
+                CK(cudaEventElapsedTime(&ms, c->ev0, c->ev1));
+                if (rep > 0 && (best[compact] == 0.f || ms < best[compact])) best[compact] = ms;
+            }
+        }
+        if (ms_full) ms_full[p] = best[0];
+        if (ms_compact) ms_compact[p] = best[1];
+        if (best[1] <= best[0] * 1.01f && live > gamma) gamma = live;  // 1 % timing noise
+    }
+    *gamma_out = gamma;
+    return HBSJD_OK;
+}
+
 int hbsjd_round(hbsjd_ctx* c, int* live_out) {
     if (!c) return HBSJD_EINVAL;
     if (!c->have_rollout) {

@@ -93,6 +93,8 @@ void launch_init_state(const State& st, const int32_t* prefix_tokens, const int3
 void launch_prefill_advance(const State& st, int S, cudaStream_t s);
 void launch_init_window(const State& st, uint32_t seed_lo, uint32_t seed_hi, cudaStream_t s);
 void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s);
+// synthetic state for the threshold calibration: the first `live` images at cursor T/2, the rest finished
+void launch_calib_state(const State& st, int live, cudaStream_t s);
 void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s);
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s);
 int accept_smem_bytes(int V);

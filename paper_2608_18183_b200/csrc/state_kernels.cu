@@ -94,6 +94,29 @@ void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s) {
     launch_k(k_export_tokens, dim3(st.B), dim3(128), 0, s, st, out);
 }
 
+__global__ void k_calib_state(State st, int live) {
+    pdl_trigger();
+    pdl_wait();
+    const int b = blockIdx.x;
+    int32_t* seq = st.seq + (size_t)b * (st.T + 1);
+    uint8_t* dl = st.delta + (size_t)b * (st.T + 1);
+    for (int t = threadIdx.x; t <= st.T; t += blockDim.x) {
+        seq[t] = 0;
+        dl[t] = 1;
+    }
+    if (threadIdx.x == 0) {
+        st.cursor[b] = b < live ? st.T / 2 : st.T;
+        st.qbase[b] = 0;
+        st.label[b] = 0;
+        st.klen[b] = 0;
+        st.pfill[b] = 0;
+    }
+}
+
+void launch_calib_state(const State& st, int live, cudaStream_t s) {
+    launch_k(k_calib_state, dim3(st.B), dim3(128), 0, s, st, live);
+}
+
 // ------------------------------------------------------------------ probability pipeline + verification
 // One CTA per (slot, window position i).  The guided logits of the position live in shared memory:
 //   guided = l_u + s (l_c - l_u); / temperature; top-k threshold by radix select (ties kept);

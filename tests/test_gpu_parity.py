@@ -237,3 +237,24 @@ def test_api_misuse_is_rejected_without_launching():
     # a weight image of the wrong size is refused
     with pytest.raises(binding.HbsjdError):
         binding.Context(w.shape, G.weights_for(w)[:-256], 4, 8)
+
+
+def test_threshold_calibration_reports_a_consistent_threshold():
+    """Sec. 4.3: a few verifier forwards in both forms pick the threshold.  Compact runs fewer rows through the
+    same page / slot tables, so it is never slower here and the calibrated threshold is the batch itself."""
+    w = synth.WORKLOADS["small_bf16"]
+    ctx = _ctx(w, max_batch=32)
+    gamma, ms_full, ms_compact = ctx.hbsjd_calibrate_gamma(32, w.window, True)
+    assert all(m > 0 for m in ms_full + ms_compact)
+    assert 0 <= gamma <= 32
+    # the reported threshold is the largest tested live count at which Compact was not slower
+    points = [32, 24, 16, 8, 4]
+    ok = [p for p, f, c in zip(points, ms_full, ms_compact) if c <= f * np.float32(1.01)]
+    assert gamma == (max(ok) if ok else 0)
+    # at a quarter of the batch Compact must win clearly (a quarter of the rows)
+    assert ms_compact[3] < ms_full[3]
+    # the context still rolls out afterwards
+    toks, k, lab = synth.make_inputs(w)
+    out, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 1, exec_mode=binding.EXEC_HYBRID, gamma=gamma))
+    assert st["committed"] == int((w.shape.T - k).sum())
+    ctx.hbsjd_destroy()
