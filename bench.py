@@ -29,8 +29,8 @@ from paper_2608_18183_b200 import synth  # noqa: E402
 
 METRIC = "committed image tokens/sec per B200 rollout; mean accepted tokens/forward"
 UNIT = "tokens/s"
-# DRAM bytes per GEMM launch (read + write) from the ncu capture summarised in
-# profiles/gemm_tcgen05_rollout_L.md: mean over the 97 GEMM launches of one Full round of workload L.
+# DRAM bytes per GEMM launch (read + write) from an ncu capture of the rollout (dram__bytes_read.sum +
+# dram__bytes_write.sum, summarised under profiles/): mean over the 97 GEMM launches of one Full round of workload L.
 NCU_GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"L": 54.9e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -174,7 +174,7 @@ def main():
     ap.add_argument("--workload", default="L", choices=sorted(synth.WORKLOADS))
     ap.add_argument("--gamma-frac", type=float, default=1.0,
                     help="Eq. 6 threshold as a fraction of the batch (Full iff live > threshold); 1.0 = the measured "
-                         "optimum, always Compact (profiles/exec_mode_and_window_sweep.md); 0 = always Full")
+                         "optimum on this implementation, always Compact; 0 = always Full")
     ap.add_argument("--exec-mode", default="hybrid", choices=["full", "compact", "hybrid"])
     ap.add_argument("--window", type=int, default=0)
     ap.add_argument("--verify", default="prob", choices=["prob", "greedy"], help="Eq. 5 (default) or Eq. 4")
