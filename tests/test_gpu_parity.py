@@ -258,3 +258,20 @@ def test_threshold_calibration_reports_a_consistent_threshold():
     out, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 1, exec_mode=binding.EXEC_HYBRID, gamma=gamma))
     assert st["committed"] == int((w.shape.T - k).sum())
     ctx.hbsjd_destroy()
+
+
+def test_window_one_probabilistic_rollout_is_the_oracle_ar_sampler():
+    """W = 1 (no drafts): every round commits one token sampled from the model's next-token distribution with
+    word 1 of (image, position, round) -- token for token the oracle's plain AR sampler (fp32 model)."""
+    w = synth.WORKLOADS["tiny"]
+    toks, k, lab = synth.make_inputs(synth.with_shape(w, prefix=("uniform", 0, 40)), seed=5)
+    ctx = _ctx(w)
+    model = O.Model(w.shape, G.weights_for(w))
+    same = 0
+    for seed in (3, 4, 5):
+        out, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, seed, window=1))
+        assert st["rejects"] == 0 and st["committed"] == st["image_forwards"] == int((w.shape.T - k).sum())
+        ar = model.ar_rollout(toks, k, lab, O.make_params(1, w.history_offset, seed=seed))
+        same += int(np.array_equal(out.cpu().numpy(), ar))
+    assert same >= 2  # fp32: a flip needs a sampling target within ~1e-6 of a bin edge
+    ctx.hbsjd_destroy()
