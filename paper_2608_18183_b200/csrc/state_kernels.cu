@@ -141,7 +141,7 @@ struct AccShared {
     unsigned int sel_prefix, sel_k;
     int result;
     uint32_t words[4];
-    float bcast;
+    int jfirst;
 };
 
 __device__ __forceinline__ unsigned int float_key(float x) {
@@ -200,22 +200,49 @@ __device__ int block_pick(const float* a, int V, uint32_t word, AccShared& sh) {
     if (S != 0) {
         const unsigned long long target = ((unsigned long long)word * S) >> 32;
         if (target >= excl && target < excl + sh.redu[wid]) {  // exactly one warp
+            // The warp walks its segment 1024 entries at a time: eight independent warp totals of 128
+            // entries each (a lane holds four consecutive entries per step) locate the step, one scan over
+            // the lanes locates the lane, and the lane resolves its four entries.
             unsigned long long run = excl;
-            for (int it = 0; it < seg; it += 32) {
-                const int v = base + it + lane;
-                const unsigned long long x = (v < V) ? fixed_weight(a[v]) : 0ull;
-                unsigned long long incl = x;
+            bool found = false;
+            for (int c0 = 0; c0 < seg && !found; c0 += 1024) {
+                auto lane_weight = [&](int k) -> unsigned long long {
+                    const int v = base + c0 + k * 128 + lane * 4;
+                    if (c0 + k * 128 >= seg || v >= V) return 0ull;
+                    const float4 e = *reinterpret_cast<const float4*>(a + v);
+                    return (unsigned long long)fixed_weight(e.x) + fixed_weight(e.y) + fixed_weight(e.z) +
+                           fixed_weight(e.w);
+                };
+                unsigned long long tot[8];
 #pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += t;
+                for (int k = 0; k < 8; ++k) tot[k] = warp_sum_u64(lane_weight(k));
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    if (found) continue;
+                    if (run + tot[k] > target) {
+                        const unsigned long long mine = lane_weight(k);
+                        unsigned long long incl = mine;
+#pragma unroll
+                        for (int o = 1; o < 32; o <<= 1) {
+                            const unsigned long long t = __shfl_up_sync(0xffffffffu, incl, o);
+                            if (lane >= o) incl += t;
+                        }
+                        const unsigned int hit = __ballot_sync(0xffffffffu, run + incl > target);
+                        if (lane == __ffs(hit) - 1) {
+                            const int v = base + c0 + k * 128 + lane * 4;
+                            unsigned long long r = run + incl - mine;
+                            int e = 0;
+                            for (; e < 3; ++e) {
+                                r += fixed_weight(a[v + e]);
+                                if (r > target) break;
+                            }
+                            sh.result = v + e;
+                        }
+                        found = true;
+                    } else {
+                        run += tot[k];
+                    }
                 }
-                const unsigned int hit = __ballot_sync(0xffffffffu, run + incl > target);
-                if (hit) {
-                    if (lane == 0) sh.result = base + it + (__ffs(hit) - 1);
-                    break;
-                }
-                run += __shfl_sync(0xffffffffu, incl, 31);
             }
         }
     }
@@ -511,7 +538,7 @@ __device__ void prob_pipeline(float* g, const float* __restrict__ lc, const floa
 }
 
 // Stand-alone probability pipeline: one CTA per row of logits.
-__global__ void __launch_bounds__(ACC_THREADS) k_probs(const float* __restrict__ lc, const float* __restrict__ lu,
+__global__ void __launch_bounds__(ACC_THREADS, 2) k_probs(const float* __restrict__ lc, const float* __restrict__ lu,
                                                        int V, float cfg_scale, float temperature, int top_k,
                                                        float* __restrict__ p) {
     pdl_trigger();
@@ -523,7 +550,7 @@ __global__ void __launch_bounds__(ACC_THREADS) k_probs(const float* __restrict__
     prob_pipeline(g, lc + row * V, lu ? lu + row * V : nullptr, V, cfg_scale, temperature, top_k, p + row * V, sh);
 }
 
-__global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArgs a) {
+__global__ void __launch_bounds__(ACC_THREADS, 2) k_prob_accept(State st, AcceptArgs a) {
     pdl_trigger();
     pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -578,7 +605,6 @@ __global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArg
     }
 
     // accept test (Eq. 5)
-    bool accept = true;
     if (!last) {
         if (tid == 0) {
             const float pz = g[z];
@@ -586,73 +612,14 @@ __global__ void __launch_bounds__(ACC_THREADS) k_prob_accept(State st, AcceptArg
             if (is_delta) alpha = pz;
             else alpha = fminf(1.0f, __fdiv_rn(pz, qrow[z]));
             const float u = (float)(sh.words[0] >> 8) * (1.0f / 16777216.0f);
-            sh.bcast = (u < alpha) ? 1.f : 0.f;
             a.flag[oidx] = (u < alpha) ? 1 : 0;
         }
-        __syncthreads();
-        accept = sh.bcast != 0.f;
     }
-    const uint32_t w1 = sh.words[1], w2 = sh.words[2];
 
-    // refreshed draft candidate ~ p_i (weight sums already in sh.redu)
-    const int ref = block_pick(g, V, w2, sh);
-    int rep = -1;
-    if (last) {
-        rep = block_pick(g, V, w1, sh);  // bonus token ~ p_{n-1}: same array, same sums
-    } else if (!accept) {
-        // residual [p - q]+ (point-mass proposal: p with z removed), overwriting p in shared memory
-        const int seg = warp_segment(V);
-        if (is_delta) {
-            if (tid == 0) {
-                sh.redu[z / seg] -= fixed_weight(g[z]);
-                g[z] = 0.f;
-            }
-        } else {
-            unsigned long long wsum = 0;
-            const int vend = min(V, (wid + 1) * seg);
-            for (int v0 = wid * seg + lane * 4; v0 < vend; v0 += 128 * 8) {
-                float4 q4[8];  // eight proposal loads in flight per thread
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    if (v0 + k * 128 < vend) q4[k] = *reinterpret_cast<const float4*>(qrow + v0 + k * 128);
-#pragma unroll
-                for (int k = 0; k < 8; ++k) {
-                    const int v = v0 + k * 128;
-                    if (v < vend) {
-                        float4 p4 = *reinterpret_cast<float4*>(g + v);
-                        p4.x = fmaxf(__fsub_rn(p4.x, q4[k].x), 0.f);
-                        p4.y = fmaxf(__fsub_rn(p4.y, q4[k].y), 0.f);
-                        p4.z = fmaxf(__fsub_rn(p4.z, q4[k].z), 0.f);
-                        p4.w = fmaxf(__fsub_rn(p4.w, q4[k].w), 0.f);
-                        *reinterpret_cast<float4*>(g + v) = p4;
-                        wsum += (unsigned long long)fixed_weight(p4.x) + fixed_weight(p4.y) + fixed_weight(p4.z) +
-                                fixed_weight(p4.w);
-                    }
-                }
-            }
-            wsum = warp_sum_u64(wsum);
-            if (lane == 0) sh.redu[wid] = wsum;
-        }
-        __syncthreads();
-        rep = block_pick(g, V, w1, sh);
-        if (rep < 0) {  // empty residual: sample p_i itself with the same word
-            unsigned long long wsum = 0;
-            for (int v = wid * seg + lane * 4; v < min(V, (wid + 1) * seg); v += 128) {
-                const float4 p4 = *reinterpret_cast<const float4*>(pout + v);
-                *reinterpret_cast<float4*>(g + v) = p4;
-                wsum += (unsigned long long)fixed_weight(p4.x) + fixed_weight(p4.y) + fixed_weight(p4.z) +
-                        fixed_weight(p4.w);
-            }
-            wsum = warp_sum_u64(wsum);
-            if (lane == 0) sh.redu[wid] = wsum;
-            __syncthreads();
-            rep = block_pick(g, V, w1, sh);
-        }
-    }
-    if (tid == 0) {
-        a.cand_ref[oidx] = ref;
-        a.cand_rep[oidx] = rep;
-    }
+    // refreshed draft candidate ~ p_i (weight sums already in sh.redu).  The replacement / bonus token is
+    // needed at one position per image only (the first reject, else the last): k_commit draws it.
+    const int ref = block_pick(g, V, sh.words[2], sh);
+    if (tid == 0) a.cand_ref[oidx] = ref;
 }
 
 int accept_smem_bytes(int V) { return V * (int)sizeof(float) + (int)sizeof(AccShared); }
@@ -673,34 +640,107 @@ void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
     launch_k(k_prob_accept, dim3(grid), dim3(ACC_THREADS), accept_smem_bytes(st.V), s, st, a);
 }
 
-// ------------------------------------------------------------------ commit + refresh (one warp per slot)
-// First reject by ballot over the accept flags; lane 0 commits the accepted prefix plus the replacement
-// (or bonus) token, advances the cursor -- the KV commit is this cursor move: entries at and after the
-// new cursor are recomputed by the next forward (Sec. 4.2 "Independent progress") -- and rebuilds the window.
-__global__ void k_commit(State st, AcceptArgs a) {
+// ------------------------------------------------------------------ commit + refresh (one CTA per slot)
+// First reject by ballot over the accept flags.  The token committed after the accepted prefix is drawn
+// here, at that one position: the replacement ~ [p_j - q]+ (point-mass proposal: p_j with the draft removed)
+// at the first reject j (Eq. 5 and the sentence after it), else the bonus token ~ p_{n-1}, both with word 1
+// of (image, position, round); the probabilities are read back from this round's p rows.  Thread 0 then
+// commits, advances the cursor -- the KV commit is this cursor move: entries at and after the new cursor are
+// recomputed by the next forward (Sec. 4.2 "Independent progress") -- and rebuilds the window.
+__global__ void __launch_bounds__(ACC_THREADS) k_commit(State st, AcceptArgs a) {
     pdl_trigger();
     pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const int slot = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-    if (slot >= a.S) return;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    float* g = (float*)smem_raw;  // [V]
+    AccShared& sh = *(AccShared*)(smem_raw + (size_t)st.V * sizeof(float));
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int slot = blockIdx.x;
     const int n = st.slot_n[slot];
     if (n == 0) return;
+    const int V = st.V;
     const int img = st.slot_img[slot], c = st.slot_c[slot];
-    int j = -1;
-    for (int base = 0; base < n - 1; base += 32) {
-        const int i = base + lane;
-        const bool rej = (i < n - 1) && (a.flag[(size_t)img * st.Wmax + i] == 0);
-        const unsigned int b = __ballot_sync(0xffffffffu, rej);
-        if (b) {
-            j = base + __ffs(b) - 1;
-            break;
-        }
-    }
-    if (lane != 0) return;
     int32_t* seq = st.seq + (size_t)img * (st.T + 1);
     uint8_t* dl = st.delta + (size_t)img * (st.T + 1);
+    if (wid == 0) {
+        int j = -1;
+        for (int base = 0; base < n - 1; base += 32) {
+            const int i = base + lane;
+            const bool rej = (i < n - 1) && (a.flag[(size_t)img * st.Wmax + i] == 0);
+            const unsigned int b = __ballot_sync(0xffffffffu, rej);
+            if (b) {
+                j = base + __ffs(b) - 1;
+                break;
+            }
+        }
+        if (lane == 0) {
+            sh.jfirst = j;
+            const int t = c + (j >= 0 ? j : n - 1) + 1;
+            philox4x32_10((uint32_t)img, (uint32_t)t, a.round, 0u, a.seed_lo, a.seed_hi, sh.words);
+        }
+    }
+    __syncthreads();
+    const int j = sh.jfirst;
     const int m = j >= 0 ? j + 1 : n;
-    const int tok = a.cand_rep[(size_t)img * st.Wmax + (m - 1)];
+    int tok;
+    if (a.greedy) {
+        if (tid != 0) return;
+        tok = a.cand_rep[(size_t)img * st.Wmax + (m - 1)];
+    } else {
+        const int is = m - 1, t = c + m;
+        const float* prow = a.pcur + ((size_t)img * st.Wmax + is) * V;
+        const bool reject = j >= 0;
+        const int z = reject ? seq[t] : -1;
+        const bool is_delta = reject && dl[t] != 0;
+        const float* qrow =
+            (reject && !is_delta) ? a.pprev + ((size_t)img * st.Wmax + (t - st.qbase[img] - 1)) * V : nullptr;
+        const int seg = warp_segment(V);
+        const int vend = min(V, (wid + 1) * seg);
+        for (int pass = 0; pass < 2; ++pass) {
+            // pass 0: the residual (or p itself for the bonus token); pass 1, only after an empty residual:
+            // p_j itself with the same word
+            unsigned long long wsum = 0;
+            for (int v0 = wid * seg + lane * 4; v0 < vend; v0 += 128 * 4) {
+                float4 p4[4], q4[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int v = v0 + k * 128;
+                    if (v < vend) {
+                        p4[k] = *reinterpret_cast<const float4*>(prow + v);
+                        if (qrow && pass == 0) q4[k] = *reinterpret_cast<const float4*>(qrow + v);
+                    }
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int v = v0 + k * 128;
+                    if (v < vend) {
+                        float4 x = p4[k];
+                        if (pass == 0) {
+                            if (qrow) {
+                                x.x = fmaxf(__fsub_rn(x.x, q4[k].x), 0.f);
+                                x.y = fmaxf(__fsub_rn(x.y, q4[k].y), 0.f);
+                                x.z = fmaxf(__fsub_rn(x.z, q4[k].z), 0.f);
+                                x.w = fmaxf(__fsub_rn(x.w, q4[k].w), 0.f);
+                            } else if (is_delta && (z >> 2) == (v >> 2)) {
+                                if ((z & 3) == 0) x.x = 0.f;
+                                if ((z & 3) == 1) x.y = 0.f;
+                                if ((z & 3) == 2) x.z = 0.f;
+                                if ((z & 3) == 3) x.w = 0.f;
+                            }
+                        }
+                        *reinterpret_cast<float4*>(g + v) = x;
+                        wsum += (unsigned long long)fixed_weight(x.x) + fixed_weight(x.y) + fixed_weight(x.z) +
+                                fixed_weight(x.w);
+                    }
+                }
+            }
+            wsum = warp_sum_u64(wsum);
+            if (lane == 0) sh.redu[wid] = wsum;
+            __syncthreads();
+            tok = block_pick(g, V, sh.words[1], sh);
+            if (tok >= 0 || !reject) break;
+        }
+        if (tid != 0) return;
+    }
     seq[c + m] = tok;
     dl[c + m] = 0;
     const int c2 = c + m;
@@ -733,7 +773,10 @@ __global__ void k_commit(State st, AcceptArgs a) {
 }
 
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s) {
-    launch_k(k_commit, dim3((a.S + 3) / 4), dim3(128), 0, s, st, a);
+    static int configured[64] = {0};
+    const int bytes = accept_smem_bytes(st.V);
+    ensure_dynamic_smem(k_commit, bytes, configured);
+    launch_k(k_commit, dim3(a.S), dim3(ACC_THREADS), bytes, s, st, a);
 }
 
 // ------------------------------------------------------------------ stand-alone verification step

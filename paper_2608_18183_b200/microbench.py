@@ -1,0 +1,202 @@
+"""Kernel-level micro-benchmarks of the rollout library, one JSON line per case.
+
+    python -m paper_2608_18183_b200.microbench accept   # verification step at a paper-like commit length
+    python -m paper_2608_18183_b200.microbench probs    # probability pipeline on 4096 rows
+    python -m paper_2608_18183_b200.microbench gemm     # decoder GEMM shapes of a workload, each timed alone
+
+The rollouts of bench.py run random-weight models whose acceptance pattern is not the paper's; `accept` feeds
+the verification kernels synthetic (p, q) pairs instead: targets p = softmax(l), proposals q = softmax(l + sigma *
+noise), drafts drawn from q, sigma tuned so that the mean number of committed tokens per image matches the
+paper's probabilistic mode (2.3 tokens per forward, Table 10), at the L workload's sizes (batch 128, guidance,
+window 32, V = 16384, top-k 1000).  Inputs are made with torch on the GPU; every timed step runs in the library.
+Times are CUDA events around single calls (each call ends with a stream synchronise, so a launch gap of a few
+microseconds is inside the figure); bandwidths divide the algorithmic bytes by that time.  `gemm` times bursts of
+20 back-to-back launches instead (the way the decoder issues them).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+
+import numpy as np
+
+
+def _median_us(torch, fn, reset=None, reps=9, warm=3):
+    ts = []
+    for i in range(warm + reps):
+        if reset is not None:
+            reset()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warm:
+            ts.append(e0.elapsed_time(e1) * 1e3)
+    return float(np.median(ts))
+
+
+def _small_context(binding, synth, vocab, max_batch, max_window):
+    """A context whose model is irrelevant here (one thin layer): the stand-alone entry points only use its
+    stream, limits and scratch."""
+    sh = synth.ModelShape(1, 64, 1, 64, vocab, 4, 4, 3, "bf16")
+    return binding.Context(sh, synth.make_weights(sh, 3, target_entropy=None), max_batch, max_window)
+
+
+def verify_inputs(torch, B, W, T, V, branches, cfg_scale, top_k, sigma, seed, sampled_frac=0.85, logit_std=2.5):
+    """Device tensors of one verification step: ragged cursors, a previous round that committed 1..3 tokens,
+    sampled drafts (with their proposal rows in q) and history drafts (point-mass proposals).  The proposals
+    are the guided, top-k filtered targets perturbed by sigma * noise in the logits."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    base = torch.randn(B, W, V, device="cuda", generator=g) * logit_std
+    if branches == 2:
+        unc = base * 0.5 + torch.randn(B, W, V, device="cuda", generator=g)
+        logits = torch.stack([base, unc]).contiguous()
+        guided = unc + cfg_scale * (base - unc)
+    else:
+        logits = base[None].contiguous()
+        guided = base
+    cursor = torch.randint(0, T - W, (B,), device="cuda", generator=g, dtype=torch.int32)
+    back = torch.randint(1, 4, (B,), device="cuda", generator=g, dtype=torch.int32)
+    qbase = torch.clamp(cursor - back, min=0)
+    seq = torch.randint(0, V, (B, T + 1), device="cuda", generator=g, dtype=torch.int32)
+    delta = torch.ones(B, T + 1, device="cuda", dtype=torch.uint8)
+    q = torch.empty(B, W, V, device="cuda")
+    cur, qb = cursor.tolist(), qbase.tolist()
+    i = torch.arange(0, W - 1, device="cuda")
+    for b in range(B):
+        shift = cur[b] - qb[b]
+        noisy = guided[b] + sigma * torch.randn(W, V, device="cuda", generator=g)
+        if 0 < top_k < V:
+            kth = torch.topk(noisy, top_k, dim=-1).values[:, -1:]
+            noisy = torch.where(noisy >= kth, noisy, torch.full_like(noisy, float("-inf")))
+        # the proposal of the draft verified at window position i sits in row i + shift of the previous
+        # round's probabilities
+        q[b] = torch.softmax(torch.roll(noisy, shift, dims=0), dim=-1)
+        draws = torch.multinomial(q[b], 1, generator=g).squeeze(1).to(torch.int32)  # one draw per proposal row
+        qi = i + shift
+        ok = (qi < W) & (torch.rand(W - 1, device="cuda", generator=g) < sampled_frac)
+        t = cur[b] + 1 + i[ok]
+        seq[b, t] = draws[qi[ok]]
+        delta[b, t] = 0
+    return logits, q, cursor, seq, delta, qbase
+
+
+def bench_accept(args):
+    import torch
+    from . import binding, synth
+    B, W, T, V, branches, top_k = args.batch, args.window, 256, args.vocab, 2 if args.cfg_scale != 1.0 else 1, args.top_k
+    ctx = _small_context(binding, synth, V, B, W)
+
+    def run_case(sigma, timed):
+        logits, q, cursor, seq, delta, qbase = verify_inputs(torch, B, W, T, V, branches, args.cfg_scale, top_k, sigma, args.seed)
+        p_out = torch.zeros(B, W, V, device="cuda")
+        m_out = torch.zeros(B, dtype=torch.int32, device="cuda")
+        desc = binding.hbsjd_verify_desc(B, W, T, V, branches, 16, 0, top_k, args.cfg_scale, 1.0, args.seed, 7, 0)
+        st = [cursor.clone(), seq.clone(), delta.clone(), qbase.clone()]
+
+        def reset():
+            st[0].copy_(cursor); st[1].copy_(seq); st[2].copy_(delta); st[3].copy_(qbase)
+
+        def call():
+            ctx.hbsjd_verify(desc, logits, q, p_out, st[0], st[1], st[2], st[3], m_out)
+
+        reset()
+        call()
+        m = m_out.float().mean().item()
+        us = _median_us(torch, call, reset) if timed else None
+        return m, us, (m_out < W).float().mean().item()
+
+    # sigma by bisection on the mean commit length (monotone decreasing in sigma)
+    lo, hi = 0.0, 8.0
+    for _ in range(10):
+        mid = 0.5 * (lo + hi)
+        m, _, _ = run_case(mid, False)
+        if m > args.target_commit:
+            lo = mid
+        else:
+            hi = mid
+    sigma = 0.5 * (lo + hi)
+    m, us, rej = run_case(sigma, True)
+    rows = B * W
+    # logits of every branch read + probabilities written; proposal rows are read only at a reject (one per
+    # image) and for the accept ratio (single elements), so they are left out of the algorithmic figure
+    alg = rows * V * 4.0 * (branches + 1)
+    print(json.dumps({"case": "accept", "batch": B, "window": W, "V": V, "branches": branches, "top_k": top_k,
+                      "sigma": round(sigma, 4), "mean_committed_per_image": round(m, 3),
+                      "images_with_reject": round(rej, 3), "us": round(us, 1),
+                      "algorithmic_bytes": alg, "GB_s": round(alg / us / 1e3, 1)}))
+    ctx.hbsjd_destroy()
+
+
+def bench_probs(args):
+    import torch
+    from . import binding, synth
+    V, rows = args.vocab, args.rows
+    ctx = _small_context(binding, synth, V, 2, 4)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(args.seed)
+    lc = torch.randn(rows, V, device="cuda", generator=g) * 3.5
+    lu = torch.randn(rows, V, device="cuda", generator=g) * 3.5
+    out = torch.empty_like(lc)
+    for name, (u, s, tau, k) in {"plain": (None, 1.0, 1.0, 0), "guidance": (lu, 4.0, 1.0, 0),
+                                 "top_k": (None, 1.0, 1.0, 1000), "guidance+top_k": (lu, 4.0, 1.0, 1000),
+                                 "guidance+top_k+temperature": (lu, 4.0, 0.7, 1000)}.items():
+        def call():
+            ctx._check(ctx.lib.hbsjd_probs(ctx.h, lc.data_ptr(), None if u is None else u.data_ptr(), rows, s, tau, k,
+                                           out.data_ptr()), "hbsjd_probs")
+        us = _median_us(torch, call)
+        alg = rows * V * 4.0 * ((2 if u is not None else 1) + 1)
+        print(json.dumps({"case": "probs", "variant": name, "rows": rows, "V": V, "us": round(us, 1),
+                          "algorithmic_bytes": alg, "GB_s": round(alg / us / 1e3, 1)}))
+    ctx.hbsjd_destroy()
+
+
+def bench_gemm(args):
+    import torch
+    os.environ.setdefault("HBSJD_GEMM_NOSYNC", "1")  # hbsjd_gemm returns without waiting: launches run back to back
+    from . import binding, synth
+    w = synth.WORKLOADS[args.workload]
+    s = w.shape
+    D, F, V = s.dim, s.ffn_hidden, s.vocab
+    M = args.rows or w.batch * (2 if w.cfg_scale != 1.0 else 1) * w.window
+    ctx = _small_context(binding, synth, 64, 2, 4)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(args.seed)
+    for name, N, K, acc in [("qkv", 3 * D, D, 0), ("attention out (+=)", D, D, 1), ("gate|up", 2 * F, D, 0),
+                            ("down (+=)", D, F, 1), ("head", V, D, 0)]:
+        A = torch.randn(M, K, device="cuda", generator=g).bfloat16()
+        Wt = (torch.randn(N, K, device="cuda", generator=g) * 0.05).bfloat16()
+        Cm = torch.zeros(M, N, device="cuda")
+        def burst():
+            for _ in range(20):
+                ctx.hbsjd_gemm(A, Wt, Cm, accumulate=bool(acc))
+        us = _median_us(torch, burst, reps=5, warm=2) / 20
+        print(json.dumps({"case": "gemm", "name": name, "M": M, "N": N, "K": K, "accumulate": acc,
+                          "us": round(us, 1), "TFLOP_s": round(2.0 * M * N * K / us / 1e6, 1)}))
+    ctx.hbsjd_destroy()
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
+    ap.add_argument("case", choices=["accept", "probs", "gemm"])
+    ap.add_argument("--workload", default="L")
+    ap.add_argument("--batch", type=int, default=128)
+    ap.add_argument("--window", type=int, default=32)
+    ap.add_argument("--vocab", type=int, default=16384)
+    ap.add_argument("--top-k", type=int, default=1000)
+    ap.add_argument("--cfg-scale", type=float, default=4.0)
+    ap.add_argument("--target-commit", type=float, default=2.3)
+    ap.add_argument("--rows", type=int, default=0)
+    ap.add_argument("--seed", type=int, default=1)
+    args = ap.parse_args(argv)
+    if args.case == "probs" and not args.rows:
+        args.rows = 4096
+    {"accept": bench_accept, "probs": bench_probs, "gemm": bench_gemm}[args.case](args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

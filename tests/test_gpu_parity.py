@@ -271,7 +271,7 @@ def test_window_one_probabilistic_rollout_is_the_oracle_ar_sampler():
     for seed in (3, 4, 5):
         out, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, seed, window=1))
         assert st["rejects"] == 0 and st["committed"] == st["image_forwards"] == int((w.shape.T - k).sum())
-        ar = model.ar_rollout(toks, k, lab, O.make_params(1, w.history_offset, seed=seed))
+        ar = model.ar_rollout(toks, k, lab, G.orc_params(w, seed, window=1))
         same += int(np.array_equal(out.cpu().numpy(), ar))
     assert same >= 2  # fp32: a flip needs a sampling target within ~1e-6 of a bin edge
     ctx.hbsjd_destroy()

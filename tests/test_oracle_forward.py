@@ -32,7 +32,7 @@ def test_forward_bf16_weights_fp32_activations_matches_torch(tiny_bf16):
     got = m.forward_full(1, seq)
     ref = TR.forward(w.shape, P, 1, seq)
     assert np.abs(got - ref).max() < 2e-5
-    # with bf16 activation rounding the result moves, but stays within the bf16 budget
+    # with bf16 activation rounding the result moves, but stays within the bf16 tolerance
     mb = O.Model(w.shape, img, act_bf16=True)
     gb = mb.forward_full(1, seq)
     d = np.abs(gb - ref).max()
