@@ -10,6 +10,8 @@
 //   * independent progress, shared cond/uncond state under CFG,
 //     replacement token = next start token, no cache repair          (Sec. 4.2, "Independent progress")
 //   * Full / Compact / Hybrid execution choice                       (Sec. 4.3, Eq. 6)
+//   * the distillation score of a completed trajectory: teacher and
+//     student full-sequence forwards and the bidirectional KL          (Eq. 3)
 //
 // Only tests, the smoke check and the benchmark's cpu_baseline leg may call
 // this file.  It shares no code, header, table or constant generator with the
@@ -28,7 +30,9 @@
 // RoPE shift invariance; softmax/top-k properties; W=1 rollout == plain AR
 // sampler; greedy SJD == greedy AR; accept/resample identity by brute force;
 // chi-square of SJD rollouts against the enumerated AR joint; Full == Compact;
-// subset independence; CFG special cases.
+// subset independence; CFG special cases; bidirectional KL closed forms (two
+// classes, equal distributions, shift invariance, symmetry) and the score
+// against the torch restatement's logits.
 // Parity unpinned: the absolute token values for a given seed (the paper
 // prints no worked example).
 
@@ -790,6 +794,72 @@ void orc_ar_rollout(void* m, int B, const int32_t* prefix_tokens, const int32_t*
         }
         for (int t = 1; t <= T; ++t) out[(size_t)b * T + t - 1] = seq[t];
     }
+}
+
+// ------------------------------------------------------- distillation score (Eq. 3)
+
+// D_biKL(p, q) = 1/2 KL(p || q) + 1/2 KL(q || p) for p = softmax(s), q = softmax(t),
+// the definition written out in the log domain, double throughout.
+double bikl_row(const float* s, const float* t, int V) {
+    double ms = s[0], mt = t[0];
+    for (int v = 1; v < V; ++v) {
+        if (s[v] > ms) ms = s[v];
+        if (t[v] > mt) mt = t[v];
+    }
+    double zs = 0.0, zt = 0.0;
+    for (int v = 0; v < V; ++v) {
+        zs += std::exp((double)s[v] - ms);
+        zt += std::exp((double)t[v] - mt);
+    }
+    const double lzs = std::log(zs), lzt = std::log(zt);
+    double kl_pq = 0.0, kl_qp = 0.0;
+    for (int v = 0; v < V; ++v) {
+        const double lp = (double)s[v] - ms - lzs, lq = (double)t[v] - mt - lzt;
+        kl_pq += std::exp(lp) * (lp - lq);
+        kl_qp += std::exp(lq) * (lq - lp);
+    }
+    return 0.5 * kl_pq + 0.5 * kl_qp;
+}
+
+void orc_bikl(const float* s, const float* t, int rows, int V, double* out) {
+    for (int r = 0; r < rows; ++r) out[r] = bikl_row(s + (size_t)r * V, t + (size_t)r * V, V);
+}
+
+// Eq. 3 on completed trajectories: for image b with real prefix k_b, the mean over t = k_b+1..T of
+// D_biKL(p_S(. | x_<t), p_T(. | x_<t)); both models see the same tokens and the image's class, no
+// guidance, no temperature, no top-k.  pos [B][T]: entry t-1 holds the term of position t (0 for t <= k_b);
+// per_image [B] (0 when k_b = T); *loss = mean of per_image over the images with k_b < T.
+void orc_score(void* student, void* teacher, int B, const int32_t* tokens, const int32_t* prefix_len,
+               const int32_t* labels, double* pos, double* per_image, double* loss) {
+    const Model& S = *(Model*)student;
+    const Model& Tm = *(Model*)teacher;
+    const int T = S.T, V = S.d.V;
+#pragma omp parallel for schedule(dynamic)
+    for (int b = 0; b < B; ++b) {
+        std::vector<int32_t> seq(T + 1, 0);
+        for (int t = 1; t <= T; ++t) seq[t] = tokens[(size_t)b * T + t - 1];
+        std::vector<float> ls((size_t)T * V), lt((size_t)T * V);
+        // inputs are sequence indices 0..T-1 (class token, x_1..x_{T-1}); output row i is the distribution of x_{i+1}
+        forward_full(S, labels[b], seq.data(), T, ls.data());
+        forward_full(Tm, labels[b], seq.data(), T, lt.data());
+        const int k = prefix_len[b];
+        double sum = 0.0;
+        for (int t = 1; t <= T; ++t) {
+            double d = 0.0;
+            if (t >= k + 1) d = bikl_row(&ls[(size_t)(t - 1) * V], &lt[(size_t)(t - 1) * V], V);
+            pos[(size_t)b * T + t - 1] = d;
+            sum += d;
+        }
+        per_image[b] = k < T ? sum / (double)(T - k) : 0.0;
+    }
+    double tot = 0.0;
+    int cnt = 0;
+    for (int b = 0; b < B; ++b)
+        if (prefix_len[b] < T) {
+            tot += per_image[b];
+            ++cnt;
+        }
+    *loss = cnt ? tot / cnt : 0.0;
 }
 
 int orc_num_threads() {

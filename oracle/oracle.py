@@ -73,6 +73,9 @@ def lib():
         L.orc_rollout_logits.argtypes = [vp, C.c_int, C.c_int, f32p]
         L.orc_rollout_stats.argtypes = [vp, C.POINTER(C.c_int64), i32p, i32p, C.c_int]
         L.orc_ar_rollout.argtypes = [vp, C.c_int, i32p, i32p, i32p, i32p, C.POINTER(Params), i32p]
+        L.orc_bikl.argtypes = [f32p, f32p, C.c_int, C.c_int, C.POINTER(C.c_double)]
+        L.orc_score.argtypes = [vp, vp, C.c_int, i32p, i32p, i32p, C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                C.POINTER(C.c_double)]
         L.orc_num_threads.restype = C.c_int
         _lib = L
     return _lib
@@ -144,6 +147,29 @@ def replay_round(V, T, W, H, greedy, seed, image_id, rnd, c, seq, delta, p, qpre
                                _p(seq, C.c_int32), _p(delta, C.c_uint8), _p(p, C.c_float), _p(qprev, C.c_float),
                                qbase, C.byref(j))
     return cc.value, m, j.value
+
+
+def bikl(s, t) -> np.ndarray:
+    """Eq. 3's divergence per row: D_biKL(softmax(s), softmax(t)) for fp32 logits [rows, V] -> float64 [rows]."""
+    s = np.ascontiguousarray(np.atleast_2d(s), dtype=np.float32)
+    t = np.ascontiguousarray(np.atleast_2d(t), dtype=np.float32)
+    assert s.shape == t.shape
+    out = np.zeros(s.shape[0], dtype=np.float64)
+    lib().orc_bikl(_p(s, C.c_float), _p(t, C.c_float), s.shape[0], s.shape[1], _p(out, C.c_double))
+    return out
+
+
+def score(student: "Model", teacher: "Model", tokens, prefix_len, labels):
+    """Eq. 3 on completed trajectories.  Returns (pos float64 [B, T], per_image float64 [B], loss)."""
+    tk, pl, lb = _i32(tokens), _i32(prefix_len), _i32(labels)
+    assert student.shape.T == teacher.shape.T and student.shape.vocab == teacher.shape.vocab
+    B, T = tk.shape
+    pos = np.zeros((B, T), dtype=np.float64)
+    per = np.zeros(B, dtype=np.float64)
+    loss = C.c_double(0.0)
+    lib().orc_score(student.h, teacher.h, B, _p(tk, C.c_int32), _p(pl, C.c_int32), _p(lb, C.c_int32),
+                    _p(pos, C.c_double), _p(per, C.c_double), C.byref(loss))
+    return pos, per, loss.value
 
 
 class Model:
