@@ -228,6 +228,31 @@ int hbsjd_verify_static(void *cuda_stream, const hbsjd_verify_desc *d, const flo
                         float *p_out, int32_t *cursor, int32_t *seq, uint8_t *delta, int32_t *qbase,
                         int32_t *m_out);
 
+/* Bidirectional KL of Eq. 3 per row: out[r] = 1/2 KL(p || q) + 1/2 KL(q || p) with p = softmax(logits_s[r]),
+ * q = softmax(logits_t[r]).  logits_s, logits_t: DEVICE fp32 [rows, V], V the context's vocabulary; out: DEVICE
+ * fp32 [rows].  fp32 arithmetic with running maxima (no overflow for any finite logits).  Runs on the context's
+ * stream and waits for completion. */
+int hbsjd_bikl(hbsjd_ctx *c, const float *logits_s, const float *logits_t, int rows, float *out);
+
+/* Distillation score of completed trajectories (Eq. 3): for image b with real prefix k_b, the mean over the
+ * generated positions t = k_b+1..T of D_biKL(p_S(. | x_<t), p_T(. | x_<t)), where both models read the same
+ * tokens and class label (no guidance, temperature 1, no top-k), then the mean over the images of the batch that
+ * generated anything (k_b < T).  This is the step that follows the rollout in the on-policy distillation loop.
+ *   student, teacher  two contexts with the same grid (T) and vocabulary; batch <= max_batch of both.  Both
+ *                     models run full-sequence causal forwards in chunks of min(max_window) inputs per image
+ *                     through the same kernels as the rollout; their rollout state and KV caches are
+ *                     overwritten (a stepped rollout cannot be continued afterwards).
+ *   tokens        DEVICE int32 [batch, T]   completed trajectories (e.g. hbsjd_rollout's out_tokens)
+ *   prefix_len    DEVICE int32 [batch]      k_b in 0..T
+ *   class_labels  DEVICE int32 [batch]
+ *   bikl_pos      DEVICE fp32 [batch, T] or NULL: entry t-1 = the term of position t (0 for t <= k_b)
+ *   per_image     DEVICE fp32 [batch] or NULL: the per-image means (0 where k_b = T)
+ *   loss          HOST float: the batch mean
+ * Work is enqueued on each context's own stream with event dependencies between them; the call returns after
+ * both streams finished.  Errors as hbsjd_rollout (arguments are validated on the host before any launch). */
+int hbsjd_score(hbsjd_ctx *student, hbsjd_ctx *teacher, int batch, const int32_t *tokens, const int32_t *prefix_len,
+                const int32_t *class_labels, float *bikl_pos, float *per_image, float *loss);
+
 /* Per-kernel-class timing with CUDA events on the context's stream (off by default).  While enabled,
  * every launch of a timed class is bracketed by an event pair; totals accumulate until the next
  * hbsjd_profile(c, 1), which also resets them.  work = algorithmic FLOPs (GEMM: 2 M N K per launch) or

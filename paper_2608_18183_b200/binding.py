@@ -17,7 +17,8 @@ EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
 EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
-           "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_strerror", "hbsjd_last_error"]
+           "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
+           "hbsjd_last_error"]
 
 
 class hbsjd_model_desc(C.Structure):
@@ -93,6 +94,8 @@ def load():
         L.hbsjd_set_state.argtypes = [vp, vp, vp, vp, vp, C.c_int32]
         L.hbsjd_debug_read.argtypes = [vp, C.c_int, C.c_int, vp, C.c_size_t]
         L.hbsjd_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int]
+        L.hbsjd_bikl.argtypes = [vp, vp, vp, C.c_int, vp]
+        L.hbsjd_score.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp, vp, C.POINTER(C.c_float)]
         L.hbsjd_strerror.argtypes = [C.c_int]
         L.hbsjd_strerror.restype = C.c_char_p
         L.hbsjd_last_error.argtypes = [vp]
@@ -259,6 +262,32 @@ class Context:
         self._check(self.lib.hbsjd_gemm(self.h, A.data_ptr(), W.data_ptr(), Cout.data_ptr(), M, N, K,
                                         1 if accumulate else 0), "hbsjd_gemm")
         return Cout
+
+    def hbsjd_bikl(self, logits_s, logits_t):
+        """Device fp32 [rows, V] logits of two models -> device fp32 [rows] bidirectional KL (Eq. 3)."""
+        out = self._torch.empty(logits_s.shape[0], dtype=self._torch.float32, device="cuda")
+        assert logits_s.shape == logits_t.shape and logits_s.is_contiguous() and logits_t.is_contiguous()
+        self._check(self.lib.hbsjd_bikl(self.h, logits_s.data_ptr(), logits_t.data_ptr(), logits_s.shape[0],
+                                        out.data_ptr()), "hbsjd_bikl")
+        return out
+
+    def hbsjd_score(self, teacher: "Context", tokens, prefix_len, class_labels):
+        """Eq. 3 on completed trajectories, this context the student.  Device int32 tensors in; returns
+        (bikl_pos device fp32 [batch, T], per_image device fp32 [batch], loss float)."""
+        torch = self._torch
+        batch = tokens.shape[0]
+        assert tokens.is_cuda and tokens.dtype == torch.int32 and tokens.is_contiguous()
+        assert tuple(tokens.shape) == (batch, self.shape.T)
+        assert prefix_len.dtype == torch.int32 and class_labels.dtype == torch.int32
+        pos = torch.empty((batch, self.shape.T), dtype=torch.float32, device="cuda")
+        per = torch.empty(batch, dtype=torch.float32, device="cuda")
+        loss = C.c_float(0.0)
+        self._check(self.lib.hbsjd_score(self.h, teacher.h, batch, tokens.data_ptr(), prefix_len.data_ptr(),
+                                         class_labels.data_ptr(), pos.data_ptr(), per.data_ptr(), C.byref(loss)),
+                    "hbsjd_score")
+        self.batch = 0
+        teacher.batch = 0
+        return pos, per, loss.value
 
     def hbsjd_destroy(self):
         if self.h:

@@ -56,6 +56,7 @@ struct hbsjd_ctx {
     // host-buffer staging
     int32_t *stage_tok, *stage_len, *stage_lab, *stage_out;
     void* verify_scratch;
+    float *score_pos, *score_img, *score_loss;  // [Bmax][T], [Bmax], [1]
     // per-class event timing
     bool profiling;
     struct ProfSlot { cudaEvent_t a, b; int cls; double work; };
@@ -320,7 +321,8 @@ void free_all(hbsjd_ctx* c) {
                     c->st.qbase, c->st.label, c->st.klen, c->st.pfill, c->st.slot_img, c->st.slot_c, c->st.slot_n,
                     c->st.counters, c->st.m_last, c->st.j_last, c->pbuf[0], c->pbuf[1], c->flag, c->cand_rep,
                     c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act,
-                    c->stage_tok, c->stage_len, c->stage_lab, c->stage_out, c->verify_scratch};
+                    c->stage_tok, c->stage_len, c->stage_lab, c->stage_out, c->verify_scratch,
+                    c->score_pos, c->score_img, c->score_loss};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->h_counters) cudaFreeHost(c->h_counters);
@@ -468,6 +470,9 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
         unsigned char* vs = nullptr;
         if ((rc = dev_alloc(c, &vs, verify_scratch_bytes(c->Bmax, c->Wmax)))) return rc;
         c->verify_scratch = vs;
+        if ((rc = dev_alloc(c, &c->score_pos, (size_t)c->Bmax * c->T))) return rc;
+        if ((rc = dev_alloc(c, &c->score_img, (size_t)c->Bmax))) return rc;
+        if ((rc = dev_alloc(c, &c->score_loss, 1))) return rc;
     }
     c->pool.resize(1024);
     for (auto& s : c->pool) {
@@ -703,6 +708,122 @@ int hbsjd_verify(hbsjd_ctx* c, const hbsjd_verify_desc* d, const float* logits, 
     const VerifyScratch sc = verify_scratch_carve(c->verify_scratch, d->batch, d->window);
     CK(verify_enqueue(vd, sc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out, c->stream));
     CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
+}
+
+int hbsjd_bikl(hbsjd_ctx* c, const float* logits_s, const float* logits_t, int rows, float* out) {
+    if (!c) return HBSJD_EINVAL;
+    if (!logits_s || !logits_t || !out || rows < 1 || c->d.vocab % 4) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_bikl: argument out of range");
+        return HBSJD_EINVAL;
+    }
+    launch_bikl_rows(logits_s, logits_t, rows, c->d.vocab, out, c->stream);
+    CK(cudaGetLastError());
+    CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
+}
+
+int hbsjd_score(hbsjd_ctx* student, hbsjd_ctx* teacher, int batch, const int32_t* tokens, const int32_t* prefix_len,
+                const int32_t* class_labels, float* bikl_pos, float* per_image, float* loss) {
+    hbsjd_ctx* c = student;  // errors are reported on the student context
+    if (!c) return HBSJD_EINVAL;
+    c->err[0] = 0;
+    if (!teacher || teacher == student || !tokens || !prefix_len || !class_labels || !loss) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_score: null argument, or one context given twice");
+        return HBSJD_EINVAL;
+    }
+    const int T = c->T, V = c->d.vocab;
+    if (teacher->T != T || teacher->d.vocab != V || teacher->d.grid_w != c->d.grid_w || V % 4 || batch < 1 ||
+        batch > c->Bmax || batch > teacher->Bmax || teacher->d.n_classes != c->d.n_classes) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_score: contexts do not match (grid, vocabulary, classes) or batch %d too large",
+                 batch);
+        return HBSJD_EINVAL;
+    }
+    // validate the integer inputs on the host before any kernel runs
+    std::vector<int32_t> hk(batch), hl(batch), ht((size_t)batch * T);
+    CK(cudaMemcpyAsync(hk.data(), prefix_len, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(hl.data(), class_labels, batch * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaMemcpyAsync(ht.data(), tokens, (size_t)batch * T * sizeof(int32_t), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    for (int b = 0; b < batch; ++b) {
+        if (hk[b] < 0 || hk[b] > T || hl[b] < 0 || hl[b] > c->d.n_classes) {
+            snprintf(c->err, sizeof(c->err), "image %d: prefix_len %d or label %d out of range", b, hk[b], hl[b]);
+            return HBSJD_EINVAL;
+        }
+        for (int t = 0; t < T; ++t)
+            if (ht[(size_t)b * T + t] < 0 || ht[(size_t)b * T + t] >= V) {
+                snprintf(c->err, sizeof(c->err), "image %d: token %d out of range", b, t);
+                return HBSJD_EINVAL;
+            }
+    }
+    const int W = c->Wmax < teacher->Wmax ? c->Wmax : teacher->Wmax;
+    float* pos = bikl_pos ? bikl_pos : c->score_pos;
+    float* img = per_image ? per_image : c->score_img;
+    hbsjd_ctx* both[2] = {student, teacher};
+    for (hbsjd_ctx* x : both) {
+        State& st = x->st;
+        st.B = batch;
+        st.T = T;
+        st.V = V;
+        st.D = x->d.dim;
+        st.Hh = x->d.n_heads;
+        st.dh = x->dh;
+        st.F = x->d.ffn_hidden;
+        st.L = x->d.n_layers;
+        st.C = x->d.n_classes;
+        st.Bmax = x->Bmax;
+        st.Wmax = x->Wmax;
+        st.W = W;
+        st.H = 1;
+        st.nb = 1;
+        x->have_rollout = false;
+        x->live = 0;
+        launch_score_init(st, tokens, class_labels, prefix_len, x == student ? pos : nullptr, x->stream);
+        x->launches++;
+    }
+    for (int done = 0; done < T; done += W) {
+        for (hbsjd_ctx* x : both) {
+            launch_setup(x->st, 1, 0, x->stream);
+            x->launches++;
+            const int rc = forward_any(x, batch, true);
+            if (rc) {
+                if (x != c) snprintf(c->err, sizeof(c->err), "teacher forward: %.200s", x->err);
+                return rc;
+            }
+            if (x->profiling) {  // fold this forward's event pairs while its byte counters are current
+                const int rs = sync_counters(x);
+                if (rs) return rs;
+            }
+        }
+        // the divergence kernel reads both models' logits on the student's stream; the teacher's next
+        // forward overwrites its logits and waits for that kernel in turn
+        CK(cudaEventRecord(teacher->ev2, teacher->stream));
+        CK(cudaStreamWaitEvent(c->stream, teacher->ev2, 0));
+        {
+            // timed with the vocabulary-wide class: 2 V floats read per input, as the byte count of that class
+            const int ps = prof_begin(c, HBSJD_PROF_ACCEPT, 0.0);
+            launch_bikl_slots(c->st, batch, c->logits, teacher->logits, prefix_len, pos, c->stream);
+            prof_end(c, ps);
+        }
+        c->launches++;
+        CK(cudaEventRecord(c->ev2, c->stream));
+        CK(cudaStreamWaitEvent(teacher->stream, c->ev2, 0));
+        for (hbsjd_ctx* x : both) {
+            launch_prefill_advance(x->st, batch, x->stream);
+            x->launches++;
+        }
+    }
+    launch_score_reduce(batch, T, prefix_len, pos, img, c->score_loss, c->stream);
+    c->launches++;
+    CK(cudaMemcpyAsync(loss, c->score_loss, sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+    CK(cudaGetLastError());
+    for (hbsjd_ctx* x : both) {
+        const int rc = sync_counters(x);
+        if (rc) {
+            if (x != c) snprintf(c->err, sizeof(c->err), "teacher: %.200s", x->err);
+            return rc;
+        }
+    }
     return HBSJD_OK;
 }
 

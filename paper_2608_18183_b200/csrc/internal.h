@@ -101,6 +101,16 @@ int accept_smem_bytes(int V);
 void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
                   float* p, cudaStream_t s);
 
+// ---- distillation score (score_kernels.cu)
+void launch_bikl_rows(const float* ls, const float* lt, int rows, int V, float* out, cudaStream_t s);
+// terms of the inputs of one scoring chunk (slot tables of st; logits rows slot * W + i of both models)
+void launch_bikl_slots(const State& st, int S, const float* ls, const float* lt, const int32_t* prefix_len,
+                       float* pos, cudaStream_t s);
+void launch_score_init(const State& st, const int32_t* tokens, const int32_t* labels, const int32_t* prefix_len,
+                       float* pos, cudaStream_t s);
+void launch_score_reduce(int B, int T, const int32_t* prefix_len, const float* pos, float* per_image, float* loss,
+                         cudaStream_t s);
+
 // ---- tcgen05 GEMM (gemm_tcgen05.cu)
 // C[M,N] fp32 (+)= A[M,K] bf16 . W[N,K]^T bf16.  force_bn: 0 = choose the tile width from the shape.
 // error_flag: device int set non-zero if a bounded pipeline wait gave up.  Returns 0, or a negative

@@ -3,6 +3,8 @@
     python -m paper_2608_18183_b200.microbench accept   # verification step at a paper-like commit length
     python -m paper_2608_18183_b200.microbench probs    # probability pipeline on 4096 rows
     python -m paper_2608_18183_b200.microbench gemm     # decoder GEMM shapes of a workload, each timed alone
+    python -m paper_2608_18183_b200.microbench bikl     # bidirectional-KL reduction (Eq. 3) on 4096 row pairs
+    python -m paper_2608_18183_b200.microbench score    # teacher/student scoring of a batch of trajectories (Eq. 3)
 
 The rollouts of bench.py run random-weight models whose acceptance pattern is not the paper's; `accept` feeds
 the verification kernels synthetic (p, q) pairs instead: targets p = softmax(l), proposals q = softmax(l + sigma *
@@ -16,6 +18,7 @@ microseconds is inside the figure); bandwidths divide the algorithmic bytes by t
 from __future__ import annotations
 
 import argparse
+import ctypes as C
 import json
 import os
 import sys
@@ -88,7 +91,7 @@ def verify_inputs(torch, B, W, T, V, branches, cfg_scale, top_k, sigma, seed, sa
 def bench_accept(args):
     import torch
     from . import binding, synth
-    B, W, T, V, branches, top_k = args.batch, args.window, 256, args.vocab, 2 if args.cfg_scale != 1.0 else 1, args.top_k
+    B, W, T, V, branches, top_k = args.batch or 128, args.window, 256, args.vocab, 2 if args.cfg_scale != 1.0 else 1, args.top_k
     ctx = _small_context(binding, synth, V, B, W)
 
     def run_case(sigma, timed):
@@ -180,11 +183,80 @@ def bench_gemm(args):
     ctx.hbsjd_destroy()
 
 
+def bench_bikl(args):
+    import torch
+    from . import binding, synth
+    V, rows = args.vocab, args.rows
+    ctx = _small_context(binding, synth, V, 2, 4)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(args.seed)
+    ls = torch.randn(rows, V, device="cuda", generator=g) * 3.0
+    lt = 0.6 * ls + torch.randn(rows, V, device="cuda", generator=g) * 2.0
+    out = torch.empty(rows, device="cuda")
+
+    def call():
+        ctx._check(ctx.lib.hbsjd_bikl(ctx.h, ls.data_ptr(), lt.data_ptr(), rows, out.data_ptr()), "hbsjd_bikl")
+    us = _median_us(torch, call)
+    alg = rows * V * 4.0 * 2
+    print(json.dumps({"case": "bikl", "rows": rows, "V": V, "us": round(us, 1), "algorithmic_bytes": alg,
+                      "GB_s": round(alg / us / 1e3, 1)}))
+    ctx.hbsjd_destroy()
+
+
+def teacher_shape(synth, s):
+    """The scoring benchmark's teacher: the XL decoder's width and depth on the student's grid and vocabulary."""
+    x = synth.WORKLOADS["XL"].shape
+    return synth.ModelShape(x.n_layers, x.dim, x.n_heads, x.ffn_hidden, s.vocab, s.grid_h, s.grid_w, s.n_classes,
+                            s.dtype)
+
+
+def bench_score(args):
+    import torch
+    from . import binding, synth
+    w = synth.WORKLOADS[args.workload]
+    s = w.shape
+    tsh = teacher_shape(synth, s)
+    B = args.batch or w.batch
+    stu = binding.Context(s, synth.make_weights(s, w.weight_seed), B, w.window)
+    tea = binding.Context(tsh, synth.make_weights(tsh, 77, target_entropy=None), B, w.window)
+    _, k, lab = synth.make_inputs(w, batch=B)
+    rng = np.random.default_rng(args.seed)
+    toks = torch.from_numpy(rng.integers(0, s.vocab, size=(B, s.T)).astype(np.int32)).cuda()
+    kd, ld = torch.from_numpy(k).cuda(), torch.from_numpy(lab).cuda()
+
+    def call():
+        stu.hbsjd_score(tea, toks, kd, ld)
+    ms = _median_us(torch, call, reps=5, warm=2) / 1e3
+    for c in (stu, tea):
+        c.lib.hbsjd_profile(c.h, 1)
+    call()
+    prof = {}
+    for name, c in (("student", stu), ("teacher", tea)):
+        pr = binding.hbsjd_kernel_profile()
+        c.lib.hbsjd_profile_read(c.h, C.byref(pr))
+        c.lib.hbsjd_profile(c.h, 0)
+        prof[name] = {"gemm_ms": round(pr.ms[0], 2), "gemm_TFLOP_s": round(pr.work[0] / max(pr.ms[0], 1e-9) / 1e9, 1),
+                      "attention_ms": round(pr.ms[1], 2),
+                      "attention_GB_s": round(pr.work[1] / max(pr.ms[1], 1e-9) / 1e6, 1),
+                      "vocab_reduce_ms": round(pr.ms[2], 2),
+                      "vocab_reduce_GB_s": round(pr.work[2] / max(pr.ms[2], 1e-9) / 1e6, 1)}
+    flops = 0.0
+    for sh in (s, tsh):
+        D, F, V = sh.dim, sh.ffn_hidden, sh.vocab
+        flops += 2.0 * (sh.n_layers * (4 * D * D + 3 * D * F) + D * V) * B * s.T
+    print(json.dumps({"case": "score", "student": args.workload, "teacher": "XL width/depth on the student's grid",
+                      "batch": B, "T": s.T, "chunk": w.window, "ms": round(ms, 2),
+                      "positions_per_s": round(B * s.T / ms * 1e3), "gemm_flops": flops,
+                      "gemm_TFLOP_s_over_the_call": round(flops / ms / 1e9, 1), "profiled_pass": prof}))
+    stu.hbsjd_destroy()
+    tea.hbsjd_destroy()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
-    ap.add_argument("case", choices=["accept", "probs", "gemm"])
+    ap.add_argument("case", choices=["accept", "probs", "gemm", "bikl", "score"])
     ap.add_argument("--workload", default="L")
-    ap.add_argument("--batch", type=int, default=128)
+    ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--window", type=int, default=32)
     ap.add_argument("--vocab", type=int, default=16384)
     ap.add_argument("--top-k", type=int, default=1000)
@@ -193,9 +265,10 @@ def main(argv=None):
     ap.add_argument("--rows", type=int, default=0)
     ap.add_argument("--seed", type=int, default=1)
     args = ap.parse_args(argv)
-    if args.case == "probs" and not args.rows:
+    if args.case in ("probs", "bikl") and not args.rows:
         args.rows = 4096
-    {"accept": bench_accept, "probs": bench_probs, "gemm": bench_gemm}[args.case](args)
+    {"accept": bench_accept, "probs": bench_probs, "gemm": bench_gemm, "bikl": bench_bikl,
+     "score": bench_score}[args.case](args)
 
 
 if __name__ == "__main__":
