@@ -239,7 +239,7 @@ int hbsjd_bikl(hbsjd_ctx *c, const float *logits_s, const float *logits_t, int r
  * tokens and class label (no guidance, temperature 1, no top-k), then the mean over the images of the batch that
  * generated anything (k_b < T).  This is the step that follows the rollout in the on-policy distillation loop.
  *   student, teacher  two contexts with the same grid (T) and vocabulary; batch <= max_batch of both.  Both
- *                     models run full-sequence causal forwards in chunks of min(max_window) inputs per image
+ *                     models run full-sequence causal forwards in chunks of min(64, 2 min(max_window)) inputs per image
  *                     through the same kernels as the rollout; their rollout state and KV caches are
  *                     overwritten (a stepped rollout cannot be continued afterwards).
  *   tokens        DEVICE int32 [batch, T]   completed trajectories (e.g. hbsjd_rollout's out_tokens)

@@ -756,7 +756,11 @@ int hbsjd_score(hbsjd_ctx* student, hbsjd_ctx* teacher, int batch, const int32_t
                 return HBSJD_EINVAL;
             }
     }
-    const int W = c->Wmax < teacher->Wmax ? c->Wmax : teacher->Wmax;
+    // inputs per image per chunk: one branch only, so the activation buffers (sized for two branches of
+    // max_window inputs) hold twice the rollout's window
+    int W = 2 * (c->Wmax < teacher->Wmax ? c->Wmax : teacher->Wmax);
+    if (W > 64) W = 64;
+    if (W > T) W = T;
     float* pos = bikl_pos ? bikl_pos : c->score_pos;
     float* img = per_image ? per_image : c->score_img;
     hbsjd_ctx* both[2] = {student, teacher};

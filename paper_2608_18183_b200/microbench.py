@@ -245,7 +245,7 @@ def bench_score(args):
         D, F, V = sh.dim, sh.ffn_hidden, sh.vocab
         flops += 2.0 * (sh.n_layers * (4 * D * D + 3 * D * F) + D * V) * B * s.T
     print(json.dumps({"case": "score", "student": args.workload, "teacher": "XL width/depth on the student's grid",
-                      "batch": B, "T": s.T, "chunk": w.window, "ms": round(ms, 2),
+                      "batch": B, "T": s.T, "chunk": min(64, 2 * w.window, s.T), "ms": round(ms, 2),
                       "positions_per_s": round(B * s.T / ms * 1e3), "gemm_flops": flops,
                       "gemm_TFLOP_s_over_the_call": round(flops / ms / 1e9, 1), "profiled_pass": prof}))
     stu.hbsjd_destroy()
