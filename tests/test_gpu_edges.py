@@ -1,0 +1,141 @@
+"""Edge and degenerate cases of the rollout on the GPU: nothing to generate, one token to generate, one image,
+one kept token, no-op guidance, temperature and history offsets the standard workloads do not use, the largest
+vocabulary of the verification kernels."""
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+from paper_2608_18183_b200 import binding, synth
+from tests import gpu_util as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _ctx(w, **kw):
+    return binding.Context(w.shape, G.weights_for(w), kw.get("max_batch", w.batch), kw.get("max_window", w.window))
+
+
+def test_nothing_or_one_token_to_generate():
+    w = synth.WORKLOADS["tiny"]
+    T = w.shape.T
+    toks, k, lab = synth.make_inputs(w)
+    ctx = _ctx(w)
+    # every image already complete: no round runs, the prefix is the result
+    kk = np.full_like(k, T)
+    out, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(kk), G.dev(lab), G.gpu_params(w, 0))
+    assert st["rounds"] == 0 and st["committed"] == 0 and st["image_forwards"] == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), toks)
+    assert ctx.hbsjd_round() == 0                     # stepping a finished rollout is a no-op
+    # one token left, a complete image and an empty prefix side by side: one round finishes the short ones
+    kk = np.array([T - 1, T, 0, T - 1], dtype=np.int32)
+    out, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(kk), G.dev(lab), G.gpu_params(w, 3, max_rounds=1))
+    cur = ctx.hbsjd_get_state()[1]
+    assert cur[0] == T and cur[1] == T and cur[3] == T and 1 <= cur[2] <= w.window
+    model = O.Model(w.shape, G.weights_for(w))
+    r = O.Rollout(model, toks, kk, lab, G.orc_params(w, 3))
+    r.round()
+    np.testing.assert_array_equal(cur, r.state()[1])
+    # the last token of an image is the bonus sample of a window of one input
+    full, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(kk), G.dev(lab), G.gpu_params(w, 3))
+    r.run()
+    np.testing.assert_array_equal(full.cpu().numpy(), r.tokens())
+    ctx.hbsjd_destroy()
+
+
+def test_single_image_and_context_larger_than_the_call():
+    w = synth.WORKLOADS["tiny"]
+    toks, k, lab = synth.make_inputs(w)
+    big = _ctx(w, max_batch=7, max_window=16)        # limits above the call's batch and window
+    one = _ctx(w, max_batch=1)
+    model = O.Model(w.shape, G.weights_for(w))
+    for b in range(2):
+        a, _ = one.hbsjd_rollout(G.dev(toks[b:b + 1]), G.dev(k[b:b + 1]), G.dev(lab[b:b + 1]), G.gpu_params(w, 5))
+        c, _ = big.hbsjd_rollout(G.dev(toks[b:b + 1]), G.dev(k[b:b + 1]), G.dev(lab[b:b + 1]), G.gpu_params(w, 5))
+        np.testing.assert_array_equal(a.cpu().numpy(), c.cpu().numpy())
+        r = O.Rollout(model, toks[b:b + 1], k[b:b + 1], lab[b:b + 1], G.orc_params(w, 5))
+        r.run()
+        np.testing.assert_array_equal(a.cpu().numpy(), r.tokens())
+    one.hbsjd_destroy()
+    big.hbsjd_destroy()
+
+
+def test_one_kept_token_makes_sampling_greedy():
+    """top-k = 1 leaves a one-hot distribution: every sample is the argmax, so the probabilistic rollout commits
+    the greedy rollout's tokens (ties of the top logit aside: none in these models)."""
+    w = synth.WORKLOADS["tiny_bf16"]
+    toks, k, lab = synth.make_inputs(w)
+    ctx = _ctx(w)
+    a, sa = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 9, top_k=1))
+    g, sg = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 9, top_k=1,
+                                                                               verify_mode=binding.VERIFY_GREEDY))
+    np.testing.assert_array_equal(a.cpu().numpy(), g.cpu().numpy())
+    assert sa["rounds"] == sg["rounds"]
+    # top-k >= V is no filter
+    x, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 9, top_k=0))
+    y, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 9, top_k=w.shape.vocab + 5))
+    np.testing.assert_array_equal(x.cpu().numpy(), y.cpu().numpy())
+    ctx.hbsjd_destroy()
+
+
+def test_guidance_with_the_null_class_is_no_guidance():
+    """With the null class as the label both branches compute the same logits, so l_u + s (l_c - l_u) = l_c bit
+    for bit and the guided rollout equals the unguided one."""
+    w = synth.WORKLOADS["tiny_bf16"]
+    toks, k, lab = synth.make_inputs(w)
+    null = np.full_like(lab, w.shape.n_classes)
+    ctx = _ctx(w)
+    a, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(null), G.gpu_params(w, 2, cfg_scale=3.5))
+    b, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(null), G.gpu_params(w, 2, cfg_scale=1.0))
+    np.testing.assert_array_equal(a.cpu().numpy(), b.cpu().numpy())
+    ctx.hbsjd_destroy()
+
+
+@pytest.mark.parametrize("temperature,history", [(0.7, 8), (1.6, 100), (1.0, 1)])
+def test_temperature_and_history_offsets_in_lockstep(temperature, history):
+    """Temperature other than 1, a history offset beyond the sequence (every history draft falls back to the
+    keyed uniform token) and the shortest offset (a draft copies its left neighbour), fp32 model, every round
+    compared with the oracle."""
+    w = synth.with_shape(synth.WORKLOADS["tiny"], temperature=temperature, history_offset=history)
+    toks, k, lab = synth.make_inputs(synth.with_shape(w, prefix=("uniform", 0, 30)))
+    model = O.Model(w.shape, G.weights_for(w))
+    ctx = _ctx(w)
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 11)
+    assert rep["max_logit_err"] <= 1e-4 and rep["max_p_err"] <= 1e-6 and rep["replay_mismatch"] == 0
+    assert rep["tokens"] == int((w.shape.T - k).sum()) and rep["same"] == rep["tokens"]
+    ctx.hbsjd_destroy()
+
+
+def test_largest_vocabulary_of_the_verification_kernels():
+    """V = 32768 (128 KB of probabilities per CTA): probability pipeline against the oracle and one bit-exact
+    verification step."""
+    import torch
+    V = 32768
+    sh = synth.ModelShape(1, 64, 1, 64, V, 4, 4, 3, "bf16")
+    ctx = binding.Context(sh, synth.make_weights(sh, 3, target_entropy=None), 6, 8)
+    rng = np.random.default_rng(0)
+    lc = (rng.normal(size=(3, V)) * 3).astype(np.float32)
+    lu = (rng.normal(size=(3, V)) * 3).astype(np.float32)
+    for kk in (0, 500):
+        p = ctx.hbsjd_probs(G.dev(lc), G.dev(lu), 2.0, 0.9, kk).cpu().numpy()
+        for r in range(3):
+            ref = O.probs(lc[r], lu[r], s=2.0, tau=0.9, k=kk)
+            np.testing.assert_array_equal(p[r] > 0, ref > 1e-37)
+            assert np.all(np.abs(p[r] - ref) <= 1e-6 + 1e-4 * ref)
+    case = G.verify_case(5, B=6, W=8, T=32, V=V, top_k=200)
+    d = {n: G.dev(case[n]) for n in ("logits", "q", "cursor", "seq", "delta", "qbase")}
+    p_out = torch.zeros_like(d["q"])
+    m_out = torch.zeros(6, dtype=torch.int32, device="cuda")
+    ctx.hbsjd_verify(G.verify_desc(case, 4, 2), d["logits"], d["q"], p_out, d["cursor"], d["seq"], d["delta"],
+                     d["qbase"], m_out)
+    p_gpu = p_out.cpu().numpy()
+    for b in range(6):
+        c = int(case["cursor"][b])
+        if c >= case["T"]:
+            continue
+        n = min(case["W"], case["T"] - c)
+        seq, dl = case["seq"][b].copy(), case["delta"][b].copy()
+        nc, m, j = O.replay_round(V, case["T"], case["W"], case["H"], False, 4, b, 2, c, seq, dl, p_gpu[b][:n],
+                                  case["q"][b], int(case["qbase"][b]))
+        assert nc == int(d["cursor"][b]) and m == int(m_out[b])
+        np.testing.assert_array_equal(seq[:nc + 1], d["seq"][b].cpu().numpy()[:nc + 1])
+    ctx.hbsjd_destroy()
