@@ -276,7 +276,27 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
     if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns();  // set-up done
-    pdl_wait();  // everything above is on-chip set-up; operands of the previous kernel are read from here on
+    // Everything above is on-chip set-up.  The weight operand W is constant for the life of the model, so the
+    // producer thread fetches the W tiles of its first stages BEFORE the grid dependency resolves (they cross
+    // HBM while the previous kernel drains); activations, outputs and slot tables are touched only after it.
+    const bool is_producer = warp == 0 && lane == 0;
+    int prefetched = 0;  // k-blocks of the first tile whose W tile is already in flight
+    if (is_producer) {
+        const int tile = unit;  // every CTA owns at least one tile
+        const int n0 = (tile % tiles_n) * BN + (PAIR ? (int)rank * (BN / 2) : 0);
+        prefetched = num_kb < cfg::STAGES ? num_kb : cfg::STAGES;
+        for (int kb = 0; kb < prefetched; ++kb) {
+            const uint32_t b_dst = tiles + kb * cfg::STAGE_BYTES + cfg::A_BYTES;
+            if (PAIR) {
+                if (rank == 0) mbar_expect_tx(full0 + 8 * kb, 2 * cfg::STAGE_BYTES);
+                tma_load_2d_pair(b_dst, &map_w, kb * BK, n0, map_to_rank(full0 + 8 * kb, 0));
+            } else {
+                mbar_expect_tx(full0 + 8 * kb, cfg::STAGE_BYTES);
+                tma_load_2d(b_dst, &map_w, kb * BK, n0, full0 + 8 * kb);
+            }
+        }
+    }
+    pdl_wait();
     if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();  // grid dependency released
 
     if (warp == 0) {
@@ -289,13 +309,20 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 bool ok = true;
                 for (int kb = 0; kb < num_kb; ++kb, ++kc) {
                     const uint32_t s = kc % cfg::STAGES, ph = (kc / cfg::STAGES) & 1u;
+                    const uint32_t a_dst = tiles + s * cfg::STAGE_BYTES;
+                    if ((int)kc < prefetched) {
+                        // first revolution of the ring: the stage is free, its barrier is armed and its W tile
+                        // is on the way; only the activation tile is missing
+                        if (PAIR) tma_load_2d_pair(a_dst, &map_a, kb * BK, m0, map_to_rank(full0 + 8 * s, 0));
+                        else tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
+                        continue;
+                    }
                     if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
                         *abort_flag = 1;
                         atomicExch(g.error_flag, 1);
                         ok = false;
                         break;
                     }
-                    const uint32_t a_dst = tiles + s * cfg::STAGE_BYTES;
                     if (PAIR) {
                         // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
                         const uint32_t lead_full = map_to_rank(full0 + 8 * s, 0);
