@@ -267,6 +267,12 @@ typedef struct {
 } hbsjd_kernel_profile;
 int hbsjd_profile(hbsjd_ctx *c, int enable);
 int hbsjd_profile_read(hbsjd_ctx *c, hbsjd_kernel_profile *out);
+/* What an event pair adds to a timed launch: an event between two kernels makes the second one start only after
+ * the first has completed, so its launch latency lies inside the bracket (in normal operation the library's
+ * kernels are launched programmatically dependent and that latency overlaps the previous kernel).  This call
+ * brackets `reps` launches of an empty kernel in the same way and returns the median bracket in microseconds;
+ * benchmarks report it beside the per-class times so that a reader can net it out. */
+int hbsjd_profile_launch_floor(hbsjd_ctx *c, int reps, float *us_out);
 
 const char *hbsjd_strerror(int code);
 const char *hbsjd_last_error(const hbsjd_ctx *c);

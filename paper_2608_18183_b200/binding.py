@@ -16,7 +16,7 @@ VERIFY_PROB, VERIFY_GREEDY = 0, 1
 EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
-EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
+EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_profile_launch_floor", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
            "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
            "hbsjd_last_error"]
 
@@ -81,6 +81,7 @@ def load():
                                          C.POINTER(hbsjd_stats)]
         L.hbsjd_profile.argtypes = [vp, C.c_int]
         L.hbsjd_profile_read.argtypes = [vp, C.POINTER(hbsjd_kernel_profile)]
+        L.hbsjd_profile_launch_floor.argtypes = [vp, C.c_int, C.POINTER(C.c_float)]
         L.hbsjd_probs.argtypes = [vp, vp, vp, C.c_int, C.c_float, C.c_float, C.c_int, vp]
         L.hbsjd_verify.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
         L.hbsjd_verify_static.argtypes = [vp, C.POINTER(hbsjd_verify_desc)] + [vp] * 8
@@ -189,6 +190,12 @@ class Context:
         self._check(self.lib.hbsjd_profile_read(self.h, C.byref(p)), "hbsjd_profile_read")
         return {n: dict(ms=p.ms[i], work=p.work[i], launches=p.launches[i]) for i, n in enumerate(PROF_CLASSES)} | {
             "dropped": p.dropped}
+
+    def hbsjd_profile_launch_floor(self, reps=200) -> float:
+        """Median event bracket of an empty kernel launch, microseconds."""
+        us = C.c_float(0.0)
+        self._check(self.lib.hbsjd_profile_launch_floor(self.h, reps, C.byref(us)), "hbsjd_profile_launch_floor")
+        return us.value
 
     def hbsjd_probs(self, logits_c, logits_u=None, cfg_scale=1.0, temperature=1.0, top_k=0):
         """Device fp32 [rows, V] logits -> device fp32 [rows, V] probabilities."""

@@ -1,4 +1,5 @@
 // C ABI of the rollout library (see include/hbsjd.h): context, host-side round loop, debug helpers.
+#include <algorithm>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -843,6 +844,32 @@ int hbsjd_profile(hbsjd_ctx* c, int enable) {
 int hbsjd_profile_read(hbsjd_ctx* c, hbsjd_kernel_profile* out) {
     if (!c || !out) return HBSJD_EINVAL;
     *out = c->prof;
+    return HBSJD_OK;
+}
+
+int hbsjd_profile_launch_floor(hbsjd_ctx* c, int reps, float* us_out) {
+    if (!c) return HBSJD_EINVAL;
+    if (!us_out || reps < 1 || reps > (int)c->pool.size()) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_profile_launch_floor: argument out of range");
+        return HBSJD_EINVAL;
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    // a kernel in front, so that every bracket starts behind a completed kernel as in a forward
+    launch_noop(c->stream);
+    for (int i = 0; i < reps; ++i) {
+        CK(cudaEventRecord(c->pool[i].a, c->stream));
+        launch_noop(c->stream);
+        CK(cudaEventRecord(c->pool[i].b, c->stream));
+    }
+    CK(cudaStreamSynchronize(c->stream));
+    std::vector<float> us(reps);
+    for (int i = 0; i < reps; ++i) {
+        float ms = 0.f;
+        CK(cudaEventElapsedTime(&ms, c->pool[i].a, c->pool[i].b));
+        us[i] = ms * 1e3f;
+    }
+    std::sort(us.begin(), us.end());
+    *us_out = us[reps / 2];
     return HBSJD_OK;
 }
 

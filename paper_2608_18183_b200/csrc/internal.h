@@ -101,6 +101,9 @@ int accept_smem_bytes(int V);
 void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
                   float* p, cudaStream_t s);
 
+// empty kernel launched like every other (timing aid, model_kernels.cu)
+void launch_noop(cudaStream_t s);
+
 // ---- distillation score (score_kernels.cu)
 void launch_bikl_rows(const float* ls, const float* lt, int rows, int V, float* out, cudaStream_t s);
 // terms of the inputs of one scoring chunk (slot tables of st; logits rows slot * W + i of both models)

@@ -74,6 +74,12 @@ void launch_setup(const State& st, int phase, int compact, cudaStream_t s) {
     launch_k(k_setup, dim3(1), dim3(1024), 0, s, st, phase, compact);
 }
 
+__global__ void k_noop() {
+    pdl_trigger();
+    pdl_wait();
+}
+void launch_noop(cudaStream_t s) { launch_k(k_noop, dim3(1), dim3(32), 0, s); }
+
 // ------------------------------------------------------------------ embedding gather
 template <typename TA>
 __global__ void k_embed(State st, int S, const TA* __restrict__ tok_emb, const TA* __restrict__ cls_emb,
