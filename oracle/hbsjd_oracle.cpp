@@ -10,6 +10,7 @@
 //   * independent progress, shared cond/uncond state under CFG,
 //     replacement token = next start token, no cache repair          (Sec. 4.2, "Independent progress")
 //   * Full / Compact / Hybrid execution choice                       (Sec. 4.3, Eq. 6)
+//   * batch-synchronous progress, the baseline of the ablation        (Sec. 5.3, Table 2)
 //   * the distillation score of a completed trajectory: teacher and
 //     student full-sequence forwards and the bidirectional KL          (Eq. 3)
 //
@@ -30,7 +31,9 @@
 // RoPE shift invariance; softmax/top-k properties; W=1 rollout == plain AR
 // sampler; greedy SJD == greedy AR; accept/resample identity by brute force;
 // chi-square of SJD rollouts against the enumerated AR joint; Full == Compact;
-// subset independence; CFG special cases; bidirectional KL closed forms (two
+// subset independence; CFG special cases; batch-synchronous progress (common
+// pace, truncation by hand, greedy exactness, chi-square of batches of three);
+// bidirectional KL closed forms (two
 // classes, equal distributions, shift invariance, symmetry) and the score
 // against the torch restatement's logits.
 // Parity unpinned: the absolute token values for a given seed (the paper
@@ -351,7 +354,8 @@ int argmax_low(const float* p, int V) {
 }
 
 struct Params {
-    int32_t window, history, top_k, verify_mode /*0 prob, 1 greedy*/, exec_mode /*0 full,1 compact,2 hybrid*/, gamma;
+    int32_t window, history, top_k, verify_mode /*0 prob, 1 greedy*/,
+        exec_mode /*0 full, 1 compact, 2 hybrid, 3 full with batch-synchronous progress*/, gamma;
     float cfg_scale, temperature;
     uint64_t seed;
 };
@@ -364,9 +368,9 @@ struct Params {
 //   qprev          previous round's probabilities; the proposal of the draft at
 //                  position t is row (t - qbase - 1)
 // Returns m (tokens committed) and the first-reject index in *j_out (-1: none).
-int decide_and_refresh(int V, int T, int W, int H, bool greedy, int& c, int32_t* seq, uint8_t* delta,
-                       const float* p, int n, const float* qprev, int qbase, const uint32_t (*words)[4],
-                       const uint32_t* w3_beyond, int* j_out) {
+// Index of the first rejected draft of the window (Eq. 4 / Eq. 5), -1 if every draft is accepted.
+int first_reject(int V, bool greedy, int c, const int32_t* seq, const uint8_t* delta, const float* p, int n,
+                 const float* qprev, int qbase, const uint32_t (*words)[4]) {
     int j = -1;
     for (int i = 0; i + 1 < n; ++i) {
         const int t = c + i + 1;
@@ -388,8 +392,23 @@ int decide_and_refresh(int V, int T, int W, int H, bool greedy, int& c, int32_t*
         }
         if (!accept) { j = i; break; }
     }
+    return j;
+}
+
+// m_limit > 0 (batch-synchronous progress, the baseline of Sec. 5.3 "Is independent progress necessary"):
+// commit at most m_limit tokens.  An image whose own verification would commit more keeps only the first
+// m_limit of its accepted drafts (no replacement token is drawn: every one of them was accepted); *j_out is
+// then -1.
+int decide_and_refresh(int V, int T, int W, int H, bool greedy, int& c, int32_t* seq, uint8_t* delta,
+                       const float* p, int n, const float* qprev, int qbase, const uint32_t (*words)[4],
+                       const uint32_t* w3_beyond, int* j_out, int m_limit = 0) {
+    int j = first_reject(V, greedy, c, seq, delta, p, n, qprev, qbase, words);
     int m, tok;
-    if (j >= 0) {
+    if (m_limit > 0 && m_limit < (j >= 0 ? j + 1 : n)) {
+        m = m_limit;
+        tok = seq[c + m];  // an accepted draft
+        j = -1;
+    } else if (j >= 0) {
         const int t = c + j + 1;
         const float* pj = p + (size_t)j * V;
         if (greedy) {
@@ -493,7 +512,8 @@ void prefill(const Rollout& R, Image& im) {
     }
 }
 
-int image_round(Rollout& R, Image& im, int* j_out) {
+// Forward of the image's window and this round's probabilities (left in im.pcur).
+void image_forward(Rollout& R, Image& im) {
     const Model& M = *R.M;
     const int T = M.T, V = M.d.V, W = R.P.window;
     const bool cfg = R.P.cfg_scale != 1.0f;
@@ -503,21 +523,50 @@ int image_round(Rollout& R, Image& im, int* j_out) {
     for (int i = 0; i < n; ++i)
         probs(&im.logc[(size_t)i * V], cfg ? &im.logu[(size_t)i * V] : nullptr, R.P.cfg_scale, R.P.temperature,
               R.P.top_k, V, &im.pcur[(size_t)i * V]);
-    std::vector<uint32_t> words((size_t)n * 4), beyond(W);
+}
+
+void image_words(const Rollout& R, const Image& im, int n, std::vector<uint32_t>& words, std::vector<uint32_t>& beyond) {
+    const int W = R.P.window;
+    words.resize((size_t)n * 4);
+    beyond.resize(W);
     for (int i = 0; i < n; ++i) words_for(R.P, im.id, im.c + i + 1, (uint32_t)R.round, &words[(size_t)i * 4]);
     for (int d = 0; d < W; ++d) {
         uint32_t w[4];
         words_for(R.P, im.id, im.c + n + 1 + d, (uint32_t)R.round, w);
         beyond[d] = w[3];
     }
+}
+
+// Tokens the image's own verification would commit this round (after image_forward).
+int image_natural_commit(const Rollout& R, const Image& im) {
+    const int T = R.M->T, V = R.M->d.V;
+    const int n = std::min(R.P.window, T - im.c);
+    std::vector<uint32_t> words, beyond;
+    image_words(R, im, n, words, beyond);
+    const int j = first_reject(V, R.P.verify_mode == 1, im.c, im.seq.data(), im.delta.data(), im.pcur.data(), n,
+                               im.pprev.data(), im.qbase, (const uint32_t (*)[4])words.data());
+    return j >= 0 ? j + 1 : n;
+}
+
+// Verification, commit and refresh after image_forward; m_limit as in decide_and_refresh.
+int image_commit(Rollout& R, Image& im, int* j_out, int m_limit) {
+    const int T = R.M->T, V = R.M->d.V, W = R.P.window;
+    const int n = std::min(W, T - im.c);
+    std::vector<uint32_t> words, beyond;
+    image_words(R, im, n, words, beyond);
     const int c_old = im.c;
     const int m = decide_and_refresh(V, T, W, R.P.history, R.P.verify_mode == 1, im.c, im.seq.data(), im.delta.data(),
                                      im.pcur.data(), n, im.pprev.data(), im.qbase,
-                                     (const uint32_t (*)[4])words.data(), beyond.data(), j_out);
+                                     (const uint32_t (*)[4])words.data(), beyond.data(), j_out, m_limit);
     im.pprev.swap(im.pcur);
     im.qbase = c_old;
     im.last_n = n;
     return m;
+}
+
+int image_round(Rollout& R, Image& im, int* j_out) {
+    image_forward(R, im);
+    return image_commit(R, im, j_out, 0);
 }
 
 }  // namespace
@@ -593,9 +642,10 @@ int orc_decide(int V, int T, int W, int H, int greedy, int32_t* c_inout, int32_t
 }
 
 // As orc_decide, with the words drawn from Philox keyed (seed; image id, position, round).
+// m_limit > 0: batch-synchronous truncation as in decide_and_refresh.
 int orc_replay_round(int V, int T, int W, int H, int greedy, uint64_t seed, int id, uint32_t round,
                      int32_t* c_inout, int32_t* seq, uint8_t* delta, const float* p, const float* qprev, int qbase,
-                     int32_t* j_out) {
+                     int32_t* j_out, int m_limit) {
     Params P{};
     P.seed = seed;
     int c = *c_inout, j = -1;
@@ -608,7 +658,7 @@ int orc_replay_round(int V, int T, int W, int H, int greedy, uint64_t seed, int 
         beyond[d] = w[3];
     }
     const int m = decide_and_refresh(V, T, W, H, greedy != 0, c, seq, delta, p, n, qprev, qbase,
-                                     (const uint32_t (*)[4])words.data(), beyond.data(), &j);
+                                     (const uint32_t (*)[4])words.data(), beyond.data(), &j, m_limit);
     *c_inout = c;
     *j_out = j;
     return m;
@@ -674,16 +724,32 @@ int orc_rollout_round(void* r, int32_t* m_out, int32_t* j_out) {
     for (auto& im : R->img) live += im.c < T;
     if (live == 0) return 0;
     // Eq. 6: Full iff A > gamma (mode affects which rows run, never the values)
-    int mode = R->P.exec_mode == 2 ? (live > R->P.gamma ? 0 : 1) : R->P.exec_mode;
+    const bool sync = R->P.exec_mode == 3;
+    int mode = R->P.exec_mode == 2 ? (live > R->P.gamma ? 0 : 1) : (sync ? 0 : R->P.exec_mode);
     R->trace_live.push_back(live);
     R->trace_mode.push_back(mode);
     long long commits = 0, rej = 0;
+    int m_limit = 0;
+    if (sync) {
+        // batch-synchronous progress: every live image advances by the smallest commit of the batch
+        std::vector<int> nat(R->B, 0);
+#pragma omp parallel for schedule(dynamic)
+        for (int b = 0; b < R->B; ++b) {
+            Image& im = R->img[b];
+            if (im.c < T) {
+                image_forward(*R, im);
+                nat[b] = image_natural_commit(*R, im);
+            }
+        }
+        for (int b = 0; b < R->B; ++b)
+            if (R->img[b].c < T && (m_limit == 0 || nat[b] < m_limit)) m_limit = nat[b];
+    }
 #pragma omp parallel for schedule(dynamic) reduction(+ : commits, rej)
     for (int b = 0; b < R->B; ++b) {
         Image& im = R->img[b];
         int m = 0, j = -1;
         if (im.c < T) {
-            m = image_round(*R, im, &j);
+            m = sync ? image_commit(*R, im, &j, m_limit) : image_round(*R, im, &j);
             commits += m;
             rej += (j >= 0);
         }

@@ -59,7 +59,7 @@ def lib():
                                  C.c_int, u32p, u32p, i32p]
         L.orc_decide.restype = C.c_int
         L.orc_replay_round.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint64, C.c_int, C.c_uint32,
-                                       i32p, i32p, u8p, f32p, f32p, C.c_int, i32p]
+                                       i32p, i32p, u8p, f32p, f32p, C.c_int, i32p, C.c_int]
         L.orc_replay_round.restype = C.c_int
         L.orc_rollout_create.argtypes = [vp, C.c_int, i32p, i32p, i32p, i32p, C.POINTER(Params)]
         L.orc_rollout_create.restype = vp
@@ -136,8 +136,9 @@ def decide(V, T, W, H, greedy, c, seq, delta, p, qprev, qbase, words, w3_beyond)
     return cc.value, m, j.value
 
 
-def replay_round(V, T, W, H, greedy, seed, image_id, rnd, c, seq, delta, p, qprev, qbase):
-    """As decide(), words drawn from the keyed generator.  Returns (new_cursor, m, j)."""
+def replay_round(V, T, W, H, greedy, seed, image_id, rnd, c, seq, delta, p, qprev, qbase, m_limit=0):
+    """As decide(), words drawn from the keyed generator.  m_limit > 0: commit at most that many tokens
+    (batch-synchronous progress).  Returns (new_cursor, m, j)."""
     cc = C.c_int32(c)
     j = C.c_int32(-1)
     p = np.ascontiguousarray(p, dtype=np.float32)
@@ -145,7 +146,7 @@ def replay_round(V, T, W, H, greedy, seed, image_id, rnd, c, seq, delta, p, qpre
     assert seq.dtype == np.int32 and delta.dtype == np.uint8
     m = lib().orc_replay_round(V, T, W, H, int(greedy), C.c_uint64(seed), image_id, C.c_uint32(rnd), C.byref(cc),
                                _p(seq, C.c_int32), _p(delta, C.c_uint8), _p(p, C.c_float), _p(qprev, C.c_float),
-                               qbase, C.byref(j))
+                               qbase, C.byref(j), int(m_limit))
     return cc.value, m, j.value
 
 
