@@ -189,7 +189,8 @@ def main():
     ap.add_argument("--gamma-frac", type=float, default=1.0,
                     help="Eq. 6 threshold as a fraction of the batch (Full iff live > threshold); 1.0 = the measured "
                          "optimum on this implementation, always Compact; 0 = always Full")
-    ap.add_argument("--exec-mode", default="hybrid", choices=["full", "compact", "hybrid"])
+    ap.add_argument("--exec-mode", default="hybrid", choices=["full", "compact", "hybrid", "sync"],
+                    help="sync = Full execution with batch-synchronous progress (the ablation baseline of Table 2)")
     ap.add_argument("--window", type=int, default=0)
     ap.add_argument("--verify", default="prob", choices=["prob", "greedy"], help="Eq. 5 (default) or Eq. 4")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -219,7 +220,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     ctx = binding.Context(w.shape, weights, w.batch, w.window)
-    mode = {"full": binding.EXEC_FULL, "compact": binding.EXEC_COMPACT, "hybrid": binding.EXEC_HYBRID}[args.exec_mode]
+    mode = {"full": binding.EXEC_FULL, "compact": binding.EXEC_COMPACT, "hybrid": binding.EXEC_HYBRID,
+            "sync": binding.EXEC_SYNC}[args.exec_mode]
     gamma = int(args.gamma_frac * w.batch)
 
     def params(seed):

@@ -43,7 +43,12 @@ enum {
 
 enum { HBSJD_DTYPE_FP32 = 0, HBSJD_DTYPE_BF16 = 1 };
 enum { HBSJD_VERIFY_PROB = 0, HBSJD_VERIFY_GREEDY = 1 };              /* Eq. 5 / Eq. 4 */
-enum { HBSJD_EXEC_FULL = 0, HBSJD_EXEC_COMPACT = 1, HBSJD_EXEC_HYBRID = 2 };  /* Sec. 4.3 */
+enum { HBSJD_EXEC_FULL = 0, HBSJD_EXEC_COMPACT = 1, HBSJD_EXEC_HYBRID = 2,  /* Sec. 4.3 */
+       /* Full execution with batch-synchronous progress: every live image advances by the smallest commit of
+        * the batch (an image that verified more keeps only that many of its accepted drafts).  The baseline of
+        * the ablation "Is independent progress necessary for batched SJD?" (Sec. 5.3, Table 2); not a mode to
+        * use for speed. */
+       HBSJD_EXEC_SYNC = 3 };
 
 typedef struct hbsjd_ctx hbsjd_ctx;
 

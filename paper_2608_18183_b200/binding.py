@@ -13,7 +13,7 @@ LIB_PATH = os.path.join(_HERE, "lib", "libhbsjd.so")
 
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 VERIFY_PROB, VERIFY_GREEDY = 0, 1
-EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID = 0, 1, 2
+EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID, EXEC_SYNC = 0, 1, 2, 3
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 
 EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_profile_launch_floor", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",

@@ -58,6 +58,7 @@ struct hbsjd_ctx {
     int32_t *stage_tok, *stage_len, *stage_lab, *stage_out;
     void* verify_scratch;
     float *score_pos, *score_img, *score_loss;  // [Bmax][T], [Bmax], [1]
+    int32_t* m_sync;                              // [1] smallest commit of the round (batch-synchronous progress)
     // per-class event timing
     bool profiling;
     struct ProfSlot { cudaEvent_t a, b; int cls; double work; };
@@ -241,7 +242,7 @@ int forward_any(hbsjd_ctx* c, int S, bool want_logits) {
 }
 
 int choose_compact(const hbsjd_ctx* c, int live) {
-    if (c->P.exec_mode == HBSJD_EXEC_FULL) return 0;
+    if (c->P.exec_mode == HBSJD_EXEC_FULL || c->P.exec_mode == HBSJD_EXEC_SYNC) return 0;
     if (c->P.exec_mode == HBSJD_EXEC_COMPACT) return 1;
     return live > c->P.gamma ? 0 : 1;  // Eq. 6
 }
@@ -288,9 +289,14 @@ int run_round(hbsjd_ctx* c) {
     a.seed_lo = (uint32_t)(c->P.seed & 0xffffffffu);
     a.seed_hi = (uint32_t)(c->P.seed >> 32);
     a.round = (uint32_t)c->round;
+    a.m_sync = c->P.exec_mode == HBSJD_EXEC_SYNC ? c->m_sync : nullptr;
     {
         const int ps = prof_begin(c, HBSJD_PROF_ACCEPT, 0.0);
         launch_prob_accept(c->st, a, c->stream);
+        if (a.m_sync) {
+            launch_sync_min(c->st, a, c->m_sync, c->stream);
+            c->launches++;
+        }
         launch_commit(c->st, a, c->stream);
         prof_end(c, ps);
     }
@@ -323,7 +329,7 @@ void free_all(hbsjd_ctx* c) {
                     c->st.counters, c->st.m_last, c->st.j_last, c->pbuf[0], c->pbuf[1], c->flag, c->cand_rep,
                     c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act,
                     c->stage_tok, c->stage_len, c->stage_lab, c->stage_out, c->verify_scratch,
-                    c->score_pos, c->score_img, c->score_loss};
+                    c->score_pos, c->score_img, c->score_loss, c->m_sync};
     for (void* p : ptrs)
         if (p) cudaFree(p);
     if (c->h_counters) cudaFreeHost(c->h_counters);
@@ -474,6 +480,7 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
         if ((rc = dev_alloc(c, &c->score_pos, (size_t)c->Bmax * c->T))) return rc;
         if ((rc = dev_alloc(c, &c->score_img, (size_t)c->Bmax))) return rc;
         if ((rc = dev_alloc(c, &c->score_loss, 1))) return rc;
+        if ((rc = dev_alloc(c, &c->m_sync, 1))) return rc;
     }
     c->pool.resize(1024);
     for (auto& s : c->pool) {
@@ -566,7 +573,7 @@ int hbsjd_rollout(hbsjd_ctx* c, int batch, const int32_t* prefix_tokens, const i
     if (batch < 1 || batch > c->Bmax || p->window < 1 || p->window > c->Wmax || p->history_offset < 1 ||
         !(p->temperature > 0.f) || !std::isfinite(p->cfg_scale) || p->top_k < 0 ||
         (p->verify_mode != HBSJD_VERIFY_PROB && p->verify_mode != HBSJD_VERIFY_GREEDY) ||
-        p->exec_mode < HBSJD_EXEC_FULL || p->exec_mode > HBSJD_EXEC_HYBRID || p->gamma < 0) {
+        p->exec_mode < HBSJD_EXEC_FULL || p->exec_mode > HBSJD_EXEC_SYNC || p->gamma < 0) {
         snprintf(c->err, sizeof(c->err), "parameter out of range (batch %d window %d)", batch, p->window);
         return HBSJD_EINVAL;
     }

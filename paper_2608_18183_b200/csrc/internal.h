@@ -46,6 +46,7 @@ struct AcceptArgs {
     float cfg_scale, temperature;
     int top_k, greedy;
     uint32_t seed_lo, seed_hi, round;
+    const int32_t* m_sync;  // batch-synchronous progress: the smallest commit of the batch (null: independent)
 };
 
 // ---- row operations (model_kernels.cu)
@@ -97,6 +98,8 @@ void launch_export_tokens(const State& st, int32_t* out, cudaStream_t s);
 void launch_calib_state(const State& st, int live, cudaStream_t s);
 void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s);
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s);
+// smallest commit over the live slots of this round, from the accept flags (batch-synchronous progress)
+void launch_sync_min(const State& st, const AcceptArgs& a, int32_t* m_sync, cudaStream_t s);
 int accept_smem_bytes(int V);
 void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
                   float* p, cudaStream_t s);

@@ -679,10 +679,18 @@ __global__ void __launch_bounds__(ACC_THREADS) k_commit(State st, AcceptArgs a) 
         }
     }
     __syncthreads();
-    const int j = sh.jfirst;
-    const int m = j >= 0 ? j + 1 : n;
+    int j = sh.jfirst;
+    int m = j >= 0 ? j + 1 : n;
     int tok;
-    if (a.greedy) {
+    // batch-synchronous progress: an image that verified more than the batch's smallest commit keeps only that
+    // many of its accepted drafts (no replacement token is drawn: the token at the new cursor was accepted)
+    const bool held_back = a.m_sync != nullptr && *a.m_sync < m;
+    if (held_back) {
+        if (tid != 0) return;
+        m = *a.m_sync;
+        j = -1;
+        tok = seq[c + m];
+    } else if (a.greedy) {
         if (tid != 0) return;
         tok = a.cand_rep[(size_t)img * st.Wmax + (m - 1)];
     } else {
@@ -772,6 +780,38 @@ __global__ void __launch_bounds__(ACC_THREADS) k_commit(State st, AcceptArgs a) 
     if (j >= 0) atomicAdd(&st.counters[CNT_REJECTS], 1);
 }
 
+// One CTA: every thread walks the accept flags of its slots; block-wide minimum of the commits.
+__global__ void k_sync_min(State st, AcceptArgs a, int32_t* __restrict__ m_sync) {
+    pdl_trigger();
+    pdl_wait();
+    __shared__ int red[32];
+    int best = 0x7fffffff;
+    for (int slot = threadIdx.x; slot < a.S; slot += blockDim.x) {
+        const int n = st.slot_n[slot];
+        if (n == 0) continue;
+        const int img = st.slot_img[slot];
+        int m = n;
+        for (int i = 0; i < n - 1; ++i)
+            if (a.flag[(size_t)img * st.Wmax + i] == 0) {
+                m = i + 1;
+                break;
+            }
+        best = min(best, m);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best = min(best, __shfl_xor_sync(0xffffffffu, best, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) best = min(best, red[w]);
+        *m_sync = best;
+    }
+}
+
+void launch_sync_min(const State& st, const AcceptArgs& a, int32_t* m_sync, cudaStream_t s) {
+    launch_k(k_sync_min, dim3(1), dim3(1024), 0, s, st, a, m_sync);
+}
+
 void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s) {
     static int configured[64] = {0};
     const int bytes = accept_smem_bytes(st.V);
@@ -838,6 +878,7 @@ cudaError_t verify_enqueue(const VerifyDesc& d, const VerifyScratch& sc, const f
     a.seed_lo = (uint32_t)(d.seed & 0xffffffffu);
     a.seed_hi = (uint32_t)(d.seed >> 32);
     a.round = d.round;
+    a.m_sync = nullptr;
     // the commit counters accumulate with atomics: they must start at zero on every call
     cudaError_t e = cudaMemsetAsync(sc.counters, 0, 8 * sizeof(int32_t), s);
     if (e != cudaSuccess) return e;

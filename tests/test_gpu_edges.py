@@ -139,3 +139,43 @@ def test_largest_vocabulary_of_the_verification_kernels():
         assert nc == int(d["cursor"][b]) and m == int(m_out[b])
         np.testing.assert_array_equal(seq[:nc + 1], d["seq"][b].cpu().numpy()[:nc + 1])
     ctx.hbsjd_destroy()
+
+
+def test_batch_synchronous_progress_matches_the_oracle():
+    """Execution mode SYNC (the baseline of the Table 2 ablation): every live image advances by the batch's
+    smallest commit.  fp32 model, every round compared with the oracle's synchronous rollout; greedy verification
+    still gives the greedy AR tokens."""
+    w = synth.WORKLOADS["tiny"]
+    T = w.shape.T
+    toks, k, lab = synth.make_inputs(synth.with_shape(w, prefix=("uniform", 0, 30)), seed=3)
+    model = O.Model(w.shape, G.weights_for(w))
+    ctx = _ctx(w)
+    for seed in (5, 6):
+        orc = O.Rollout(model, toks, k, lab, G.orc_params(w, seed, exec_mode=3))
+        ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab),
+                          G.gpu_params(w, seed, exec_mode=binding.EXEC_SYNC, max_rounds=0))
+        rounds = 0
+        while orc.live():
+            before = ctx.hbsjd_get_state()[1].copy()
+            ctx.hbsjd_round()
+            _, m_o, _ = orc.round()
+            _, cur, seq, _, _ = ctx.hbsjd_get_state()
+            _, o_cur, o_seq, _, _ = orc.state()
+            live = before < T
+            assert len(set((cur - before)[live].tolist())) == 1        # one pace for the whole batch
+            np.testing.assert_array_equal(cur, o_cur)
+            for b in range(len(k)):
+                np.testing.assert_array_equal(seq[b, :cur[b] + 1], o_seq[b, :o_cur[b] + 1])
+            rounds += 1
+        out_sync, st_sync = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab),
+                                              G.gpu_params(w, seed, exec_mode=binding.EXEC_SYNC))
+        out_free, st_free = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab),
+                                              G.gpu_params(w, seed, exec_mode=binding.EXEC_FULL))
+        assert st_sync["rounds"] == rounds            # (more rounds than independent progress on average, not per seed)
+        assert st_sync["committed"] == st_free["committed"] == int((T - k).sum())
+        assert st_sync["compact_rounds"] == 0
+    g, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab),
+                             G.gpu_params(w, 0, exec_mode=binding.EXEC_SYNC, verify_mode=binding.VERIFY_GREEDY))
+    ar = model.ar_rollout(toks, k, lab, G.orc_params(w, 0, greedy=True, window=1))
+    np.testing.assert_array_equal(g.cpu().numpy(), ar)
+    ctx.hbsjd_destroy()
