@@ -1,7 +1,7 @@
 // bf16 decoder GEMMs on the 5th-generation tensor cores: acc[M,N] = A[M,K] . W[N,K]^T with fused epilogues.
 //
 // Both operands are K-major (activations row-major [M,K], weights row-major [N,K]).  The kernel is
-// persistent and warp-specialised: one CTA per SM walks a static list of 128 x BN output tiles;
+// persistent and warp-specialised: one CTA (or CTA pair) per SM walks a static list of 128 x BN output tiles;
 //   warp 0 (one lane)  TMA producer: 128 x 64 (A) and BN x 64 (W) bf16 tiles, 128-byte swizzle, STAGES-deep ring
 //   warp 1 (one lane)  issues tcgen05.mma (M = 128, N = BN, K = 16) into one of two TMEM accumulators
 //   warps 2..5         epilogue: tcgen05.ld of the finished accumulator while the next tile's main loop runs
@@ -14,8 +14,12 @@
 //             SWIGLU out bf16[M, N/2] = silu(acc[2f]) * acc[2f+1]   (gate/up rows interleaved at load time)
 //             QKV    2D RoPE on q and k, bf16 q[M, D], k and v written to the row's KV pages
 //
+// Large problems run 256 x 256 tiles on CTA pairs (clusters of two, cta_group::2 MMAs; see Cfg below).  The
+// weight tiles of a CTA's first ring revolution are requested before the grid dependency resolves.
+//
 // Every mbarrier wait is bounded (about a second): after the limit the kernel raises the error flag, all
-// roles leave their loops, TMEM is freed and the kernel returns.  No cluster launch, no multicast.
+// roles leave their loops, TMEM is freed and the kernel returns.  No multicast loads anywhere (the only
+// multicast is tcgen05.commit arriving on both CTAs of a pair).
 #include <cuda.h>
 
 #include <cstdio>
