@@ -1,7 +1,9 @@
-"""Checks at the benchmark's full size (workload L: 24 layers, dim 1024, vocabulary 16384, batch 128 with
-guidance = 256 physical rows, window 32 -> 8192 token rows per forward, the launch configuration bench.py times).
+"""Checks at full size: workload L (24 layers, dim 1024, vocabulary 16384, batch 128 with guidance = 256 physical
+rows, window 32 -> 8192 token rows per forward, the launch configuration bench.py times) and the other full-size
+configurations B (12 layers, no guidance), XL (36 layers, 24 x 24 tokens) and stress (L shape, batch 256, bimodal
+prefix lengths).
 
-The oracle needs about half a minute per image-round at this size, so element-wise parity is taken on sampled
+The oracle needs up to half a minute per image-round at these sizes, so element-wise parity is taken on sampled
 outputs: one image (the one with the shortest prefix) is followed in lockstep for two rounds while the GPU runs
 the whole batch shape; everything else is checked through properties that hold at any size."""
 import numpy as np
@@ -14,9 +16,9 @@ from tests import gpu_util as G
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def big():
-    w = synth.WORKLOADS["L"]
+@pytest.fixture(scope="module", params=["L", "B", "XL", "stress"])
+def big(request):
+    w = synth.WORKLOADS[request.param]
     weights = G.weights_for(w)
     ctx = binding.Context(w.shape, weights, w.batch, w.window)
     toks, k, lab = synth.make_inputs(w)
