@@ -99,7 +99,7 @@ def sample_plan(w, k):
     work per step.  The large models take the images with the shortest prefixes (cheapest pre-filling)."""
     order = [int(i) for i in np.argsort(k, kind="stable")]
     n_img, n_rounds = {"tiny": (w.batch, 0), "tiny_bf16": (w.batch, 0), "small_bf16": (w.batch, 0), "B": (4, 3),
-                       "L": (1, 1), "XL": (1, 1), "stress": (1, 1)}.get(w.name, (1, 1))
+                       "L": (1, 2), "XL": (1, 1), "stress": (1, 2)}.get(w.name, (1, 1))
     ids = list(range(n_img)) if n_img == w.batch else order[:n_img]
     what = (f"{n_img} image(s) of the batch with the shortest prefixes (ids {ids}, prefix lengths "
             f"{[int(k[i]) for i in ids]}): prefix pre-filling + {n_rounds or 'all'} rounds")
