@@ -195,7 +195,10 @@ template <int BN, bool PAIR = false>
 struct Cfg {
     // as many stages as fit beside the 32 KB epilogue staging: small tiles are latency-bound (one TMA round
     // trip per ring revolution), so a narrow tile gets a deep ring
-    static constexpr int STAGES = PAIR ? 6 : (BN >= 256 ? 4 : (BN == 128 ? 6 : (BN == 64 ? 8 : 9)));
+    static constexpr int STAGES = PAIR ? 6 : (BN >= 256 ? 4 : (BN == 128 ? 6 : 8));
+    // k-blocks that share one full / empty barrier pair (one wait and one commit per 2 x 4 MMAs)
+    static constexpr int KG = (!PAIR && BN <= 64) ? 4 : 2;
+    static constexpr int GROUPS = STAGES / KG;
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -284,19 +287,20 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     // producer thread fetches the W tiles of its first stages BEFORE the grid dependency resolves (they cross
     // HBM while the previous kernel drains); activations, outputs and slot tables are touched only after it.
     const bool is_producer = warp == 0 && lane == 0;
-    int prefetched = 0;  // k-blocks of the first tile whose W tile is already in flight
+    const int num_groups = (num_kb + cfg::KG - 1) / cfg::KG;  // barrier groups per tile
+    int prefetched = 0;  // groups of the first tile whose W tiles are already in flight
     if (is_producer) {
         const int tile = unit;  // every CTA owns at least one tile
         const int n0 = (tile % tiles_n) * BN + (PAIR ? (int)rank * (BN / 2) : 0);
-        prefetched = num_kb < cfg::STAGES ? num_kb : cfg::STAGES;
-        for (int kb = 0; kb < prefetched; ++kb) {
-            const uint32_t b_dst = tiles + kb * cfg::STAGE_BYTES + cfg::A_BYTES;
-            if (PAIR) {
-                if (rank == 0) mbar_expect_tx(full0 + 8 * kb, 2 * cfg::STAGE_BYTES);
-                tma_load_2d_pair(b_dst, &map_w, kb * BK, n0, map_to_rank(full0 + 8 * kb, 0));
-            } else {
-                mbar_expect_tx(full0 + 8 * kb, cfg::STAGE_BYTES);
-                tma_load_2d(b_dst, &map_w, kb * BK, n0, full0 + 8 * kb);
+        prefetched = num_groups < cfg::GROUPS ? num_groups : cfg::GROUPS;
+        for (int gi = 0; gi < prefetched; ++gi) {
+            const int kb0 = gi * cfg::KG;
+            const int nk = num_kb - kb0 < cfg::KG ? num_kb - kb0 : cfg::KG;
+            if (!PAIR || rank == 0) mbar_expect_tx(full0 + 8 * gi, (PAIR ? 2 : 1) * nk * cfg::STAGE_BYTES);
+            for (int k = 0; k < nk; ++k) {
+                const uint32_t b_dst = tiles + (gi * cfg::KG + k) * cfg::STAGE_BYTES + cfg::A_BYTES;
+                if (PAIR) tma_load_2d_pair(b_dst, &map_w, (kb0 + k) * BK, n0, map_to_rank(full0 + 8 * gi, 0));
+                else tma_load_2d(b_dst, &map_w, (kb0 + k) * BK, n0, full0 + 8 * gi);
             }
         }
     }
@@ -306,37 +310,37 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            uint32_t kc = 0;
+            uint32_t gc = 0;  // barrier groups issued so far
             for (int tile = unit; tile < num_tiles; tile += units) {
                 const int m0 = (tile / tiles_n) * TM + (int)rank * BM;
                 const int n0 = (tile % tiles_n) * BN + (PAIR ? (int)rank * (BN / 2) : 0);
                 bool ok = true;
-                for (int kb = 0; kb < num_kb; ++kb, ++kc) {
-                    const uint32_t s = kc % cfg::STAGES, ph = (kc / cfg::STAGES) & 1u;
-                    const uint32_t a_dst = tiles + s * cfg::STAGE_BYTES;
-                    if ((int)kc < prefetched) {
-                        // first revolution of the ring: the stage is free, its barrier is armed and its W tile
-                        // is on the way; only the activation tile is missing
-                        if (PAIR) tma_load_2d_pair(a_dst, &map_a, kb * BK, m0, map_to_rank(full0 + 8 * s, 0));
-                        else tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
-                        continue;
+                for (int kb0 = 0; kb0 < num_kb; kb0 += cfg::KG, ++gc) {
+                    const int nk = num_kb - kb0 < cfg::KG ? num_kb - kb0 : cfg::KG;
+                    const uint32_t gs = gc % cfg::GROUPS, ph = (gc / cfg::GROUPS) & 1u;
+                    const uint32_t bar = PAIR ? map_to_rank(full0 + 8 * gs, 0) : full0 + 8 * gs;
+                    const bool first_rev = (int)gc < prefetched;
+                    // first revolution of the ring: the stages are free, the barrier is armed and the W tiles
+                    // are on the way; only the activation tiles are missing
+                    if (!first_rev) {
+                        if (!mbar_wait(empty0 + 8 * gs, ph ^ 1u, abort_flag)) {
+                            *abort_flag = 1;
+                            atomicExch(g.error_flag, 1);
+                            ok = false;
+                            break;
+                        }
+                        // in a pair both CTAs' loads complete on the leader's barrier, which expects the bytes of both
+                        if (!PAIR || rank == 0) mbar_expect_tx(full0 + 8 * gs, (PAIR ? 2 : 1) * nk * cfg::STAGE_BYTES);
                     }
-                    if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
-                        *abort_flag = 1;
-                        atomicExch(g.error_flag, 1);
-                        ok = false;
-                        break;
-                    }
-                    if (PAIR) {
-                        // both CTAs' loads complete on the leader's barrier, which expects the bytes of both
-                        const uint32_t lead_full = map_to_rank(full0 + 8 * s, 0);
-                        if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * cfg::STAGE_BYTES);
-                        tma_load_2d_pair(a_dst, &map_a, kb * BK, m0, lead_full);
-                        tma_load_2d_pair(a_dst + cfg::A_BYTES, &map_w, kb * BK, n0, lead_full);
-                    } else {
-                        mbar_expect_tx(full0 + 8 * s, cfg::STAGE_BYTES);
-                        tma_load_2d(a_dst, &map_a, kb * BK, m0, full0 + 8 * s);
-                        tma_load_2d(a_dst + cfg::A_BYTES, &map_w, kb * BK, n0, full0 + 8 * s);
+                    for (int k = 0; k < nk; ++k) {
+                        const uint32_t a_dst = tiles + (gs * cfg::KG + k) * cfg::STAGE_BYTES;
+                        if (PAIR) {
+                            tma_load_2d_pair(a_dst, &map_a, (kb0 + k) * BK, m0, bar);
+                            if (!first_rev) tma_load_2d_pair(a_dst + cfg::A_BYTES, &map_w, (kb0 + k) * BK, n0, bar);
+                        } else {
+                            tma_load_2d(a_dst, &map_a, (kb0 + k) * BK, m0, bar);
+                            if (!first_rev) tma_load_2d(a_dst + cfg::A_BYTES, &map_w, (kb0 + k) * BK, n0, bar);
+                        }
                     }
                 }
                 if (!ok) break;
@@ -346,34 +350,36 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0 && rank == 0) {  // in a pair only the leader issues
             constexpr uint32_t idesc = umma_idesc(BN, TM);
-            uint32_t kc = 0, j = 0;
+            uint32_t gc = 0, j = 0;
             for (int tile = unit; tile < num_tiles; tile += units, ++j) {
                 const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
                 bool ok = mbar_wait(acce0 + 8 * buf, aph ^ 1u, abort_flag);  // epilogue drained this accumulator
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + buf * BN;
-                for (int kb = 0; kb < num_kb && ok; ++kb, ++kc) {
-                    const uint32_t s = kc % cfg::STAGES, ph = (kc / cfg::STAGES) & 1u;
-                    if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) {
+                for (int kb0 = 0; kb0 < num_kb && ok; kb0 += cfg::KG, ++gc) {
+                    const int nk = num_kb - kb0 < cfg::KG ? num_kb - kb0 : cfg::KG;
+                    const uint32_t gs = gc % cfg::GROUPS, ph = (gc / cfg::GROUPS) & 1u;
+                    if (!mbar_wait(full0 + 8 * gs, ph, abort_flag)) {
                         ok = false;
                         break;
                     }
-                    if (tl && kc == 0) tl[3] = globaltimer_ns();  // first operands landed
+                    if (tl && gc == 0) tl[3] = globaltimer_ns();  // first operands landed
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_src = tiles + s * cfg::STAGE_BYTES;
-                    const uint32_t b_src = a_src + cfg::A_BYTES;
+                    for (int kk = 0; kk < nk; ++kk) {
+                        const uint32_t a_src = tiles + (gs * cfg::KG + kk) * cfg::STAGE_BYTES;
+                        const uint32_t b_src = a_src + cfg::A_BYTES;
 #pragma unroll
-                    for (int k = 0; k < BK / 16; ++k) {
-                        if (PAIR)
-                            umma_f16_pair(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc,
-                                          (kb | k) != 0 ? 1u : 0u);
-                        else
-                            umma_f16(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc,
-                                     (kb | k) != 0 ? 1u : 0u);
+                        for (int k = 0; k < BK / 16; ++k) {
+                            const uint32_t acc = (kb0 | kk | k) != 0 ? 1u : 0u;
+                            if (PAIR)
+                                umma_f16_pair(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc, acc);
+                            else
+                                umma_f16(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc, acc);
+                        }
                     }
-                    // frees the stage (in both CTAs of a pair) once these MMAs have read it
-                    if (PAIR) umma_commit_pair(empty0 + 8 * s);
-                    else umma_commit(empty0 + 8 * s);
+                    // frees the group's stages (in both CTAs of a pair) once these MMAs have read them
+                    if (PAIR) umma_commit_pair(empty0 + 8 * gs);
+                    else umma_commit(empty0 + 8 * gs);
                 }
                 if (!ok) {
                     *abort_flag = 1;
