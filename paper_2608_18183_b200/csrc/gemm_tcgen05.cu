@@ -732,10 +732,11 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
 }  // namespace
 
 // Tile width by a small cost model: waves of tiles over the SMs times the time of one tile.  Measured with the
-// phase stamps of this kernel (HBSJD_GEMM_TIMELINE): a k-block of four dependent MMAs into one accumulator
-// takes about 0.285 us however narrow the tile is (the accumulation chain is latency-bound below N = 128..256)
-// and 0.51 us at N = 256; the epilogue adds about 0.15 us per 32 columns.  Large problems end up with 256
-// (CTA pairs), small ones with the widest tile that still fits one wave.
+// phase stamps of this kernel (HBSJD_GEMM_TIMELINE): a k-block costs about 0.47 us at N = 256 (MMA rate) and no
+// less than about 0.19 us however narrow the tile is -- there the ring of operand stages is what limits it (the
+// 16 KB activation tile of every k-block has to cross from L2 whatever N is, and about 160 KB can be in flight
+// per SM); the epilogue adds about 0.15 us per 32 columns.  Large problems end up with 256 (CTA pairs), small
+// ones with the widest tile that still fits one wave.
 int gemm_tcgen05_tile_n(int M, int N, int K) {
     const long tiles_m = (M + BM - 1) / BM;
     const int sms = 148, num_kb = K / BK;
@@ -747,7 +748,7 @@ int gemm_tcgen05_tile_n(int M, int N, int K) {
         if (N % bn != 0) continue;
         const long tiles = tiles_m * (N / bn);
         const long waves = (tiles + sms - 1) / sms;
-        const float per_kb = fmaxf(0.285f, 0.51f * (float)bn / 256.0f);  // microseconds
+        const float per_kb = fmaxf(0.19f, 0.47f * (float)bn / 256.0f);  // microseconds
         const float cost = (float)waves * (1.0f + 0.15f * (float)(bn / 32) + (float)num_kb * per_kb);
         if (best == 0 || cost < best_cost * 0.98f) {  // prefer the wider tile on a tie
             best = bn;
