@@ -527,7 +527,8 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     const int dh = m->dim / m->n_heads;
     if (dh != 16 && dh != 32 && dh != 64 && dh != 128) return HBSJD_EINVAL;
     if (m->dim % 16 || m->ffn_hidden % 16) return HBSJD_EINVAL;
-    if (m->dtype == HBSJD_DTYPE_BF16 && (m->dim % 64 || m->ffn_hidden % 64 || m->vocab % 64 || dh < 32))
+    // the fused QKV epilogue holds the cos/sin of at most 32 rotation pairs per row (head sizes 32 and 64)
+    if (m->dtype == HBSJD_DTYPE_BF16 && (m->dim % 64 || m->ffn_hidden % 64 || m->vocab % 64 || (dh != 32 && dh != 64)))
         return HBSJD_EINVAL;
     int ndev = 0;
     if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return HBSJD_ECUDA;

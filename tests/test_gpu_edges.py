@@ -179,3 +179,23 @@ def test_batch_synchronous_progress_matches_the_oracle():
     ar = model.ar_rollout(toks, k, lab, G.orc_params(w, 0, greedy=True, window=1))
     np.testing.assert_array_equal(g.cpu().numpy(), ar)
     ctx.hbsjd_destroy()
+
+
+def test_bf16_model_with_head_size_32_and_unsupported_head_sizes():
+    """Head size 32 in bf16 runs the fused QKV epilogue with half a rotation table per head and the plain attention
+    kernel; head size 128 is refused for bf16 models at creation."""
+    sh = synth.ModelShape(2, 128, 4, 256, 512, 6, 6, 5, "bf16")          # dh = 32
+    w = synth.Workload("dh32", sh, 3, 8, 2.0, 40, 1.0, 6, ("uniform", 0, 12))
+    img = synth.make_weights(sh, 9)
+    toks, k, lab = synth.make_inputs(w)
+    ctx = binding.Context(sh, img, w.batch, w.window)
+    model = O.Model(sh, img)
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 3)
+    std, tol = G.bf16_logit_tol(rep["logit_std"], sh.n_layers)
+    assert rep["max_logit_err"] <= tol and rep["abs_err_sum"] / rep["abs_err_n"] <= std
+    assert rep["max_p_err"] <= 1e-6 and rep["replay_mismatch"] == 0
+    assert rep["same"] >= 0.9 * rep["tokens"]
+    ctx.hbsjd_destroy()
+    bad = synth.ModelShape(1, 256, 2, 256, 512, 4, 4, 5, "bf16")         # dh = 128
+    with pytest.raises(binding.HbsjdError):
+        binding.Context(bad, synth.make_weights(bad, 9, target_entropy=None), 2, 4)
