@@ -101,7 +101,8 @@ typedef struct {
  *   max_batch    largest batch of hbsjd_rollout; max_window largest params.window (<= 64)
  *   cuda_stream  cudaStream_t as void*
  * Constraints: dim % n_heads == 0; head size 16/32/64/128 for fp32 models, 32 or 64 for bf16 models (64 runs
- * the tensor-core attention kernel, 32 a plain one); dim, ffn_hidden, vocab multiples of 64 for bf16.
+ * the tensor-core attention kernel, 32 a plain one); dim, ffn_hidden, vocab multiples of 64 for bf16;
+ * vocab <= 32768 (a position's probabilities stay in one CTA's shared memory).
  * Errors: HBSJD_EINVAL, HBSJD_ENOMEM, HBSJD_ECUDA. */
 int hbsjd_create(hbsjd_ctx **out, const hbsjd_model_desc *m, const void *weights, size_t weight_bytes,
                  int max_batch, int max_window, void *cuda_stream);

@@ -520,7 +520,7 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     *out = nullptr;
     if (!m || !weights) return HBSJD_EINVAL;
     if (m->n_layers < 1 || m->dim < 16 || m->n_heads < 1 || m->dim % m->n_heads != 0 || m->ffn_hidden < 16 ||
-        m->vocab < 4 || m->vocab % 4 != 0 || m->grid_h < 1 || m->grid_w < 1 || m->n_classes < 1 ||
+        m->vocab < 4 || m->vocab % 4 != 0 || m->vocab > 32768 || m->grid_h < 1 || m->grid_w < 1 || m->n_classes < 1 ||
         (m->dtype != HBSJD_DTYPE_FP32 && m->dtype != HBSJD_DTYPE_BF16) || !(m->rms_eps > 0) || !(m->rope_base > 1) ||
         max_batch < 1 || max_window < 1 || max_window > 64)
         return HBSJD_EINVAL;

@@ -283,7 +283,8 @@ void launch_hpc(const State& st, int S, int layer, const bf16* q, KvView kv, bf1
 }  // namespace
 
 bool attention_mma_supported(const State& st, const KvView& kv) {
-    return st.dh == DH && st.W <= 64 && kv.page % KB == 0 && st.Hh % 2 == 0;
+    // (the kernel keeps at most 32 page-table entries of a row in shared memory)
+    return st.dh == DH && st.W <= 64 && kv.page % KB == 0 && st.Hh % 2 == 0 && kv.pages_per_row <= 32;
 }
 
 void launch_attention_mma(const State& st, int S, int layer, const bf16* q, KvView kv, bf16* out, cudaStream_t s) {
