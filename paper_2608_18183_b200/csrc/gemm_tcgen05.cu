@@ -350,6 +350,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0 && rank == 0) {  // in a pair only the leader issues
             constexpr uint32_t idesc = umma_idesc(BN, TM);
+            const uint64_t desc_a0 = umma_desc(tiles);  // A tile of stage 0; every other operand tile by offset
             uint32_t gc = 0, j = 0;
             for (int tile = unit; tile < num_tiles; tile += units, ++j) {
                 const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
@@ -365,17 +366,19 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     }
                     if (tl && gc == 0) tl[3] = globaltimer_ns();  // first operands landed
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    // descriptors by increments of the 14-bit start-address field (16-byte units; the ring lies
+                    // below 256 KB, so the field never carries): + STAGE_BYTES per k-block, + 32 bytes per MMA
+                    uint64_t da = desc_a0 + (uint64_t)(gs * cfg::KG * (cfg::STAGE_BYTES >> 4));
+                    uint64_t db = da + (uint64_t)(cfg::A_BYTES >> 4);
                     for (int kk = 0; kk < nk; ++kk) {
-                        const uint32_t a_src = tiles + (gs * cfg::KG + kk) * cfg::STAGE_BYTES;
-                        const uint32_t b_src = a_src + cfg::A_BYTES;
 #pragma unroll
                         for (int k = 0; k < BK / 16; ++k) {
                             const uint32_t acc = (kb0 | kk | k) != 0 ? 1u : 0u;
-                            if (PAIR)
-                                umma_f16_pair(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc, acc);
-                            else
-                                umma_f16(tmem_d, umma_desc(a_src + k * 32), umma_desc(b_src + k * 32), idesc, acc);
+                            if (PAIR) umma_f16_pair(tmem_d, da + 2 * k, db + 2 * k, idesc, acc);
+                            else umma_f16(tmem_d, da + 2 * k, db + 2 * k, idesc, acc);
                         }
+                        da += (uint64_t)(cfg::STAGE_BYTES >> 4);
+                        db += (uint64_t)(cfg::STAGE_BYTES >> 4);
                     }
                     // frees the group's stages (in both CTAs of a pair) once these MMAs have read them
                     if (PAIR) umma_commit_pair(empty0 + 8 * gs);
