@@ -176,7 +176,9 @@ int hbsjd_debug_read(hbsjd_ctx *c, int what, int index, void *host_dst, size_t m
 /* Decoder GEMM as used by the round (Sec. 4.2 verifier forward): C[M,N] (+)= A[M,K] . W[N,K]^T on the
  * context's stream.  A, W: DEVICE, element type of the context (bf16: tcgen05 tensor cores, fp32
  * accumulation; fp32: CUDA cores).  C: DEVICE fp32 [M,N]; accumulate != 0 adds into C.
- * M may be any size; bf16 needs N % 64 == 0 and K % 64 == 0; A, W 16-byte aligned. */
+ * M may be any size; bf16 needs N % 64 == 0 and K % 64 == 0; A, W 16-byte aligned.  W is treated as a constant:
+ * the kernel starts fetching it before earlier work of the stream has finished, so it must not be the output of a
+ * library call still in flight on that stream (outputs of other kernels on the stream are ordered as usual). */
 int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate);
 
 /* Probability pipeline of the verification step on caller-supplied logits (Sec. 4.2: "verification uses the
