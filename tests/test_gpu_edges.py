@@ -199,3 +199,27 @@ def test_bf16_model_with_head_size_32_and_unsupported_head_sizes():
     bad = synth.ModelShape(1, 256, 2, 256, 512, 4, 4, 5, "bf16")         # dh = 128
     with pytest.raises(binding.HbsjdError):
         binding.Context(bad, synth.make_weights(bad, 9, target_entropy=None), 2, 4)
+
+
+def test_images_do_not_depend_on_their_batch_mates():
+    """Each image advances on its own: replacing the other images of the batch (here: marking them complete, or
+    giving them other prefixes and labels) leaves an image's tokens unchanged (bf16 model, guidance, top-k)."""
+    w = synth.WORKLOADS["tiny_bf16"]
+    T = w.shape.T
+    toks, k, lab = synth.make_inputs(w)
+    ctx = _ctx(w)
+    ref, _ = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 4))
+    ref = ref.cpu().numpy()
+    keep = [0, 2]
+    k2, lab2, toks2 = k.copy(), lab.copy(), toks.copy()
+    for b in range(w.batch):
+        if b not in keep:
+            k2[b] = T if b % 2 else max(0, int(k[b]) - 3)
+            lab2[b] = (lab[b] + 1) % w.shape.n_classes
+            toks2[b] = (toks[b] + 7) % w.shape.vocab
+    for mode in (binding.EXEC_FULL, binding.EXEC_COMPACT):
+        out, _ = ctx.hbsjd_rollout(G.dev(toks2), G.dev(k2), G.dev(lab2), G.gpu_params(w, 4, exec_mode=mode))
+        out = out.cpu().numpy()
+        for b in keep:
+            np.testing.assert_array_equal(out[b], ref[b])
+    ctx.hbsjd_destroy()
