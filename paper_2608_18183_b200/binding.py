@@ -68,9 +68,13 @@ _lib = None
 
 
 def load():
-    """Loads the library (no CUDA call is made).  Raises if it has not been built."""
+    """Loads the library (no CUDA call is made); compiles it first if it has not been built.  Raises if that fails."""
     global _lib
     if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            # a fresh checkout: compile in-tree (nvcc, sm_100a); there is no other implementation to fall back to
+            from . import build
+            build.build()
         if not os.path.exists(LIB_PATH):
             raise FileNotFoundError(f"{LIB_PATH} is missing: run paper_2608_18183_b200/build.py (nvcc, sm_100a)")
         L = C.CDLL(LIB_PATH)

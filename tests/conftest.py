@@ -12,6 +12,16 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """Both shared libraries are compiled before any test runs (a no-op when they are up to date): the CUDA
+    library needs only nvcc, not a GPU."""
+    from paper_2608_18183_b200 import build
+    from oracle import oracle as O
+    build.build()
+    O.build()
+
+
 _cache = {}
 
 
