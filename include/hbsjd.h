@@ -169,9 +169,24 @@ int hbsjd_set_state(hbsjd_ctx *c, const int32_t *cursor, const int32_t *seq, con
  *   HBSJD_DBG_PROBS   index = image: fp32 [window, V] probabilities of the last round
  *   HBSJD_DBG_LOGITS  index = 2*image + branch (0 conditional, 1 unconditional): fp32 [window, V]
  *   HBSJD_DBG_SLOTS   index ignored: int32 [3, n_slots] = image, cursor, n of each physical slot; returns n_slots
+ *   After hbsjd_debug_forward (index = 2*image + branch; elements of the context's type unless stated):
+ *   HBSJD_DBG_ACT_A   [n, dim]  normed operand of the last projection that ran (QKV at stage 0, gate/up at stage 1)
+ *   HBSJD_DBG_ACT_Q   [n, dim]  rotated queries        HBSJD_DBG_ACT_O  [n, dim]  attention output
+ *   HBSJD_DBG_ACT_FFN [n, ffn_hidden]  silu(gate) * up  HBSJD_DBG_ACT_H  fp32 [n, dim]  residual stream
+ *   HBSJD_DBG_KV_K / HBSJD_DBG_KV_V  [cursor + n, dim]  cache rows of sequence indices 0..cursor+n-1 of that layer;
+ *                     returns cursor + n
  * Returns the number of leading rows that are valid (or n_slots), or a negative error. */
-enum { HBSJD_DBG_PROBS = 0, HBSJD_DBG_LOGITS = 1, HBSJD_DBG_SLOTS = 2 };
+enum { HBSJD_DBG_PROBS = 0, HBSJD_DBG_LOGITS = 1, HBSJD_DBG_SLOTS = 2, HBSJD_DBG_ACT_A = 3, HBSJD_DBG_ACT_Q = 4,
+       HBSJD_DBG_ACT_O = 5, HBSJD_DBG_ACT_FFN = 6, HBSJD_DBG_ACT_H = 7, HBSJD_DBG_KV_K = 8, HBSJD_DBG_KV_V = 9 };
 int hbsjd_debug_read(hbsjd_ctx *c, int what, int index, void *host_dst, size_t max_bytes);
+
+/* Component-parity aid: runs the verifier forward of the current rollout state (Full layout, Sec. 4.2 "Batched
+ * verification") up to and including layer `layer` -- stage 0: through the attention sub-block (norm, QKV + RoPE +
+ * KV write, attention, output projection into the residual stream); stage 1: the whole block -- and stops, so
+ * that hbsjd_debug_read can fetch that layer's intermediates.  No logits, no verification; the rollout state
+ * is untouched (the KV rows written are the ones the next round rewrites with the same values).
+ * Errors: HBSJD_ESTATE without a preceding hbsjd_rollout; HBSJD_EINVAL for layer / stage out of range. */
+int hbsjd_debug_forward(hbsjd_ctx *c, int layer, int stage);
 
 /* Decoder GEMM as used by the round (Sec. 4.2 verifier forward): C[M,N] (+)= A[M,K] . W[N,K]^T on the
  * context's stream.  A, W: DEVICE, element type of the context (bf16: tcgen05 tensor cores, fp32

@@ -1,10 +1,10 @@
 """Kernel-level micro-benchmarks of the rollout library, one JSON line per case.
 
-    python -m paper_2608_18183_b200.microbench accept   # verification step at a paper-like commit length
-    python -m paper_2608_18183_b200.microbench probs    # probability pipeline on 4096 rows
-    python -m paper_2608_18183_b200.microbench gemm     # decoder GEMM shapes of a workload, each timed alone
-    python -m paper_2608_18183_b200.microbench bikl     # bidirectional-KL reduction (Eq. 3) on 4096 row pairs
-    python -m paper_2608_18183_b200.microbench score    # teacher/student scoring of a batch of trajectories (Eq. 3)
+    python microbench.py accept   # verification step at a paper-like commit length
+    python microbench.py probs    # probability pipeline on 4096 rows
+    python microbench.py gemm     # decoder GEMM shapes of a workload, each timed alone
+    python microbench.py bikl     # bidirectional-KL reduction (Eq. 3) on 4096 row pairs
+    python microbench.py score    # teacher/student scoring of a batch of trajectories (Eq. 3)
 
 The rollouts of bench.py run random-weight models whose acceptance pattern is not the paper's; `accept` feeds
 the verification kernels synthetic (p, q) pairs instead: targets p = softmax(l), proposals q = softmax(l + sigma *
@@ -24,6 +24,8 @@ import os
 import sys
 
 import numpy as np
+
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 
 
 def _median_us(torch, fn, reset=None, reps=9, warm=3):
@@ -90,7 +92,7 @@ def verify_inputs(torch, B, W, T, V, branches, cfg_scale, top_k, sigma, seed, sa
 
 def bench_accept(args):
     import torch
-    from . import binding, synth
+    from paper_2608_18183_b200 import binding, synth
     B, W, T, V, branches, top_k = args.batch or 128, args.window, 256, args.vocab, 2 if args.cfg_scale != 1.0 else 1, args.top_k
     ctx = _small_context(binding, synth, V, B, W)
 
@@ -137,7 +139,7 @@ def bench_accept(args):
 
 def bench_probs(args):
     import torch
-    from . import binding, synth
+    from paper_2608_18183_b200 import binding, synth
     V, rows = args.vocab, args.rows
     ctx = _small_context(binding, synth, V, 2, 4)
     g = torch.Generator(device="cuda")
@@ -161,7 +163,7 @@ def bench_probs(args):
 def bench_gemm(args):
     import torch
     os.environ.setdefault("HBSJD_GEMM_NOSYNC", "1")  # hbsjd_gemm returns without waiting: launches run back to back
-    from . import binding, synth
+    from paper_2608_18183_b200 import binding, synth
     w = synth.WORKLOADS[args.workload]
     s = w.shape
     D, F, V = s.dim, s.ffn_hidden, s.vocab
@@ -185,7 +187,7 @@ def bench_gemm(args):
 
 def bench_bikl(args):
     import torch
-    from . import binding, synth
+    from paper_2608_18183_b200 import binding, synth
     V, rows = args.vocab, args.rows
     ctx = _small_context(binding, synth, V, 2, 4)
     g = torch.Generator(device="cuda")
@@ -212,7 +214,7 @@ def teacher_shape(synth, s):
 
 def bench_score(args):
     import torch
-    from . import binding, synth
+    from paper_2608_18183_b200 import binding, synth
     w = synth.WORKLOADS[args.workload]
     s = w.shape
     tsh = teacher_shape(synth, s)

@@ -102,6 +102,10 @@ struct Model {
     Desc d;
     int T, dh;
     int act_bf16;
+    // Diagnostics only (noise-floor calibration; never a comparison target):
+    int acc_f32 = 0;      // dot products and sums of squares accumulate in fp32 instead of double
+    int attn_w_bf16 = 0;  // the unnormalised attention weights are rounded to bf16 before they multiply the values
+                          // (the usual tensor-core formulation; the normaliser keeps the unrounded weights)
     std::vector<float> tok_emb, cls_emb, g_out, w_head;
     std::vector<Layer> layers;
 };
@@ -119,29 +123,43 @@ size_t load_tensor(const Desc& d, const uint8_t* img, size_t off, size_t count, 
     return (off + 255) / 256 * 256;
 }
 
-// Y[n][N] = X[n][K] . W[N][K]^T, every output a double sum over k in increasing k.
-void matmul(const float* X, int n, int K, const float* W, int N, float* Y) {
-    std::vector<double> Xt((size_t)K * n);
+// Y[n][N] = X[n][K] . W[N][K]^T, every output a sum over k in increasing k, accumulated in Acc (double; float
+// only for the noise-floor diagnostic).  Output columns are spread over the host threads unless the caller already
+// runs one image per thread; an output's own sum is the same either way.
+template <typename Acc>
+void matmul_acc(const float* X, int n, int K, const float* W, int N, float* Y) {
+    std::vector<Acc> Xt((size_t)K * n);
     for (int i = 0; i < n; ++i)
-        for (int k = 0; k < K; ++k) Xt[(size_t)k * n + i] = X[(size_t)i * K + k];
+        for (int k = 0; k < K; ++k) Xt[(size_t)k * n + i] = (Acc)X[(size_t)i * K + k];
 #pragma omp parallel for schedule(static) if (!omp_in_parallel() && (size_t)N * K * n > 200000)
     for (int o = 0; o < N; ++o) {
-        std::vector<double> acc(n, 0.0);
+        std::vector<Acc> acc(n, (Acc)0);
         const float* w = W + (size_t)o * K;
         for (int k = 0; k < K; ++k) {
-            const double wk = w[k];
-            const double* xr = &Xt[(size_t)k * n];
+            const Acc wk = (Acc)w[k];
+            const Acc* xr = &Xt[(size_t)k * n];
             for (int i = 0; i < n; ++i) acc[i] += wk * xr[i];
         }
         for (int i = 0; i < n; ++i) Y[(size_t)i * N + o] = (float)acc[i];
     }
 }
 
+void matmul(const Model& M, const float* X, int n, int K, const float* W, int N, float* Y) {
+    if (M.acc_f32) matmul_acc<float>(X, n, K, W, N, Y);
+    else matmul_acc<double>(X, n, K, W, N, Y);
+}
+
 // out = x * rsqrt(mean(x^2) + eps) * g
 void rmsnorm(const Model& M, const float* x, const float* g, float* out) {
     const int D = M.d.D;
     double ss = 0.0;
-    for (int k = 0; k < D; ++k) ss += (double)x[k] * x[k];
+    if (M.acc_f32) {
+        float sf = 0.0f;
+        for (int k = 0; k < D; ++k) sf += x[k] * x[k];
+        ss = sf;
+    } else {
+        for (int k = 0; k < D; ++k) ss += (double)x[k] * x[k];
+    }
     const double r = 1.0 / std::sqrt(ss / D + (double)M.d.eps);
     for (int k = 0; k < D; ++k) {
         float v = (float)((double)x[k] * r * (double)g[k]);
@@ -177,26 +195,63 @@ void embed(const Model& M, int label, const int32_t* seq, int s, float* x) {
     for (int k = 0; k < D; ++k) x[k] = e[k];
 }
 
-void ffn_block(const Model& M, const Layer& Ly, std::vector<float>& x, int n) {
+// Copies of one layer's intermediates of forward_window, for component parity tests (any pointer may be null).
+// Row i belongs to sequence index c + i.
+struct Trace {
+    int32_t layer;
+    float* a;       // [n][D]  normed input of the QKV projection
+    float* q;       // [n][D]  rotated queries
+    float* k;       // [n][D]  rotated keys as cached
+    float* v;       // [n][D]  values as cached
+    float* o;       // [n][D]  attention output
+    float* x_attn;  // [n][D]  residual stream after the attention sub-block
+    float* m;       // [n][D]  normed input of the gate/up projection
+    float* act;     // [n][F]  silu(gate) * up
+    float* x_out;   // [n][D]  residual stream after the block
+};
+
+inline void trace_copy(float* dst, const float* src, size_t count) {
+    if (dst) std::memcpy(dst, src, count * sizeof(float));
+}
+
+// FFN sub-block in two stages: m = RMSNorm(x; g_ffn) (bf16), act = silu(W1 m) * (W3 m) (bf16); x += W2 act.
+void stage_ffn_act(const Model& M, const Layer& Ly, const float* x, int n, float* m, float* act) {
     const int D = M.d.D, F = M.d.F;
-    std::vector<float> m((size_t)n * D), gu((size_t)n * 2 * F), act((size_t)n * F), y((size_t)n * D);
+    std::vector<float> gu((size_t)n * 2 * F);
     for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], Ly.g_ffn.data(), &m[(size_t)i * D]);
-    matmul(m.data(), n, D, Ly.w_13.data(), 2 * F, gu.data());
+    matmul(M, m, n, D, Ly.w_13.data(), 2 * F, gu.data());
     for (int i = 0; i < n; ++i)
         for (int f = 0; f < F; ++f) {
             const double g = gu[(size_t)i * 2 * F + f], u = gu[(size_t)i * 2 * F + F + f];
             const double silu = g / (1.0 + std::exp(-g));
             act[(size_t)i * F + f] = maybe_bf16(M, (float)(silu * u));
         }
-    matmul(act.data(), n, F, Ly.w_2.data(), D, y.data());
+}
+
+void stage_ffn_down(const Model& M, const Layer& Ly, const float* act, int n, float* x) {
+    const int D = M.d.D, F = M.d.F;
+    std::vector<float> y((size_t)n * D);
+    matmul(M, act, n, F, Ly.w_2.data(), D, y.data());
     for (size_t k = 0; k < (size_t)n * D; ++k) x[k] = x[k] + y[k];
+}
+
+void ffn_block(const Model& M, const Layer& Ly, std::vector<float>& x, int n, const Trace* tr = nullptr) {
+    const int D = M.d.D, F = M.d.F;
+    std::vector<float> m((size_t)n * D), act((size_t)n * F);
+    stage_ffn_act(M, Ly, x.data(), n, m.data(), act.data());
+    stage_ffn_down(M, Ly, act.data(), n, x.data());
+    if (tr) {
+        trace_copy(tr->m, m.data(), (size_t)n * D);
+        trace_copy(tr->act, act.data(), (size_t)n * F);
+        trace_copy(tr->x_out, x.data(), (size_t)n * D);
+    }
 }
 
 void head(const Model& M, const std::vector<float>& x, int n, float* logits) {
     const int D = M.d.D;
     std::vector<float> hn((size_t)n * D);
     for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], M.g_out.data(), &hn[(size_t)i * D]);
-    matmul(hn.data(), n, D, M.w_head.data(), M.d.V, logits);
+    matmul(M, hn.data(), n, D, M.w_head.data(), M.d.V, logits);
 }
 
 // Attention of one query vector q (head h) at sequence index s over keys 0..s
@@ -209,7 +264,13 @@ void attend(const Model& M, const float* q, const float* K, const float* V, int 
     for (int t = 0; t <= s; ++t) {
         const float* k = K + (size_t)t * D + h * dh;
         double dot = 0.0;
-        for (int e = 0; e < dh; ++e) dot += (double)q[e] * (double)k[e];
+        if (M.acc_f32) {
+            float df = 0.0f;
+            for (int e = 0; e < dh; ++e) df += q[e] * k[e];
+            dot = df;
+        } else {
+            for (int e = 0; e < dh; ++e) dot += (double)q[e] * (double)k[e];
+        }
         sc[t] = dot * scale;
         mx = std::max(mx, sc[t]);
     }
@@ -217,12 +278,54 @@ void attend(const Model& M, const float* q, const float* K, const float* V, int 
     for (int t = 0; t <= s; ++t) {
         sc[t] = std::exp(sc[t] - mx);
         den += sc[t];
+        if (M.attn_w_bf16) sc[t] = bf16_round((float)sc[t]);
     }
     for (int e = 0; e < dh; ++e) {
         double acc = 0.0;
-        for (int t = 0; t <= s; ++t) acc += sc[t] * (double)V[(size_t)t * D + h * dh + e];
+        if (M.acc_f32) {
+            float af = 0.0f;
+            for (int t = 0; t <= s; ++t) af += (float)sc[t] * V[(size_t)t * D + h * dh + e];
+            acc = af;
+        } else {
+            for (int t = 0; t <= s; ++t) acc += sc[t] * (double)V[(size_t)t * D + h * dh + e];
+        }
         out[e] = maybe_bf16(M, (float)(acc / den));
     }
+}
+
+// Attention sub-block in three stages, rows i = 0..n-1 at sequence indices c+i.
+// (1) a = RMSNorm(x; g_attn) (bf16); qkv[i] = [q | k | v] = W_qkv a, q and k rotated by the 2D RoPE of index
+//     c+i, all three rounded (bf16): q is the query operand, k and v are the cache contents.
+void stage_qkv(const Model& M, const Layer& Ly, const float* x, int n, int c, float* a, float* qkv) {
+    const int D = M.d.D, dh = M.dh, Hh = M.d.Hh;
+    for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], Ly.g_attn.data(), &a[(size_t)i * D]);  // (bf16)
+    matmul(M, a, n, D, Ly.w_qkv.data(), 3 * D, qkv);
+    for (int i = 0; i < n; ++i) {
+        float* q = &qkv[(size_t)i * 3 * D];
+        float* k = q + D;
+        for (int h = 0; h < Hh; ++h) {
+            rope2d(M, q + h * dh, c + i);
+            rope2d(M, k + h * dh, c + i);
+        }
+        for (int e = 0; e < 3 * D; ++e) q[e] = maybe_bf16(M, q[e]);  // (bf16) query operand, cache contents
+    }
+}
+
+// (2) o[i] = causal attention of query i (row stride ldq) over keys 0..c+i of K, V laid out [idx][D]   (bf16)
+void stage_attend(const Model& M, const float* q, size_t ldq, const float* Kl, const float* Vl, int c, int n,
+                  float* o) {
+    const int D = M.d.D, dh = M.dh, Hh = M.d.Hh;
+    for (int i = 0; i < n; ++i)
+        for (int h = 0; h < Hh; ++h)
+            attend(M, q + (size_t)i * ldq + h * dh, Kl, Vl, h, c + i, &o[(size_t)i * D + h * dh]);
+}
+
+// (3) x += W_o o
+void stage_attn_out(const Model& M, const Layer& Ly, const float* o, int n, float* x) {
+    const int D = M.d.D;
+    std::vector<float> y((size_t)n * D);
+    matmul(M, o, n, D, Ly.w_o.data(), D, y.data());
+    for (size_t k = 0; k < (size_t)n * D; ++k) x[k] = x[k] + y[k];
 }
 
 // Windowed forward with a per-row KV cache (Sec. 4.2, "Batched verification").
@@ -231,38 +334,33 @@ void attend(const Model& M, const float* q, const float* K, const float* V, int 
 // 0..c-1 must be valid; entries c..c+n-1 are (over)written.  If logits != null
 // it receives [n][V] (position i predicts the token at sequence index c+i+1).
 void forward_window(const Model& M, float* kc, float* vc, int label, const int32_t* seq, int c, int n,
-                    float* logits) {
-    const int D = M.d.D, T = M.T, dh = M.dh, Hh = M.d.Hh;
-    std::vector<float> x((size_t)n * D), a((size_t)n * D), qkv((size_t)n * 3 * D), o((size_t)n * D),
-        y((size_t)n * D);
+                    float* logits, const Trace* trace = nullptr) {
+    const int D = M.d.D, T = M.T;
+    std::vector<float> x((size_t)n * D), a((size_t)n * D), qkv((size_t)n * 3 * D), o((size_t)n * D);
     for (int i = 0; i < n; ++i) embed(M, label, seq, c + i, &x[(size_t)i * D]);
     for (int l = 0; l < M.d.L; ++l) {
         const Layer& Ly = M.layers[l];
         float* Kl = kc + (size_t)l * T * D;
         float* Vl = vc + (size_t)l * T * D;
-        for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], Ly.g_attn.data(), &a[(size_t)i * D]);  // (bf16)
-        matmul(a.data(), n, D, Ly.w_qkv.data(), 3 * D, qkv.data());
-        for (int i = 0; i < n; ++i) {
-            const int s = c + i;
-            float* q = &qkv[(size_t)i * 3 * D];
-            float* k = q + D;
-            float* v = k + D;
-            for (int h = 0; h < Hh; ++h) {
-                rope2d(M, q + h * dh, s);
-                rope2d(M, k + h * dh, s);
-            }
-            for (int e = 0; e < D; ++e) {
-                q[e] = maybe_bf16(M, q[e]);                      // (bf16) query operand
-                Kl[(size_t)s * D + e] = maybe_bf16(M, k[e]);     // (bf16) cache contents
-                Vl[(size_t)s * D + e] = maybe_bf16(M, v[e]);
-            }
+        stage_qkv(M, Ly, x.data(), n, c, a.data(), qkv.data());
+        for (int i = 0; i < n; ++i) {  // the window's keys and values enter the cache before attention reads it
+            std::memcpy(Kl + (size_t)(c + i) * D, &qkv[(size_t)i * 3 * D + D], D * sizeof(float));
+            std::memcpy(Vl + (size_t)(c + i) * D, &qkv[(size_t)i * 3 * D + 2 * D], D * sizeof(float));
         }
-        for (int i = 0; i < n; ++i)
-            for (int h = 0; h < Hh; ++h)
-                attend(M, &qkv[(size_t)i * 3 * D + h * dh], Kl, Vl, h, c + i, &o[(size_t)i * D + h * dh]);  // (bf16)
-        matmul(o.data(), n, D, Ly.w_o.data(), D, y.data());
-        for (size_t k = 0; k < (size_t)n * D; ++k) x[k] = x[k] + y[k];
-        ffn_block(M, Ly, x, n);
+        stage_attend(M, qkv.data(), (size_t)3 * D, Kl, Vl, c, n, o.data());
+        stage_attn_out(M, Ly, o.data(), n, x.data());
+        const Trace* tr = (trace && trace->layer == l) ? trace : nullptr;
+        if (tr) {
+            trace_copy(tr->a, a.data(), (size_t)n * D);
+            for (int i = 0; i < n; ++i) {
+                if (tr->q) std::memcpy(tr->q + (size_t)i * D, &qkv[(size_t)i * 3 * D], D * sizeof(float));
+                if (tr->k) std::memcpy(tr->k + (size_t)i * D, Kl + (size_t)(c + i) * D, D * sizeof(float));
+                if (tr->v) std::memcpy(tr->v + (size_t)i * D, Vl + (size_t)(c + i) * D, D * sizeof(float));
+            }
+            trace_copy(tr->o, o.data(), (size_t)n * D);
+            trace_copy(tr->x_attn, x.data(), (size_t)n * D);
+        }
+        ffn_block(M, Ly, x, n, tr);
     }
     if (logits) head(M, x, n, logits);
 }
@@ -277,7 +375,7 @@ void forward_full(const Model& M, int label, const int32_t* seq, int len, float*
     for (int l = 0; l < M.d.L; ++l) {
         const Layer& Ly = M.layers[l];
         for (int s = 0; s < len; ++s) rmsnorm(M, &x[(size_t)s * D], Ly.g_attn.data(), &a[(size_t)s * D]);
-        matmul(a.data(), len, D, Ly.w_qkv.data(), 3 * D, qkv.data());
+        matmul(M, a.data(), len, D, Ly.w_qkv.data(), 3 * D, qkv.data());
         for (int s = 0; s < len; ++s) {
             float* q = &qkv[(size_t)s * 3 * D];
             for (int h = 0; h < Hh; ++h) {
@@ -293,7 +391,7 @@ void forward_full(const Model& M, int label, const int32_t* seq, int len, float*
         for (int s = 0; s < len; ++s)
             for (int h = 0; h < Hh; ++h)
                 attend(M, &qkv[(size_t)s * 3 * D + h * dh], K.data(), V.data(), h, s, &o[(size_t)s * D + h * dh]);
-        matmul(o.data(), len, D, Ly.w_o.data(), D, y.data());
+        matmul(M, o.data(), len, D, Ly.w_o.data(), D, y.data());
         for (size_t k = 0; k < (size_t)len * D; ++k) x[k] = x[k] + y[k];
         ffn_block(M, Ly, x, len);
     }
@@ -622,6 +720,41 @@ void orc_forward_window(void* m, float* kc, float* vc, int label, const int32_t*
     forward_window(*(Model*)m, kc, vc, label, seq, c, n, logits);
 }
 
+// As orc_forward_window, also copying the intermediates of layer tr->layer (component parity tests).
+void orc_forward_window_trace(void* m, float* kc, float* vc, int label, const int32_t* seq, int c, int n,
+                              float* logits, const Trace* tr) {
+    forward_window(*(Model*)m, kc, vc, label, seq, c, n, logits, tr);
+}
+
+// Single stages of one decoder block on caller-supplied inputs (component parity tests feed them the GPU's own
+// intermediates, so that each kernel is compared on identical inputs).  Same functions as forward_window runs.
+void orc_stage_qkv(void* m, int layer, const float* x, int n, int c, float* a, float* qkv) {
+    const Model& M = *(Model*)m;
+    stage_qkv(M, M.layers[layer], x, n, c, a, qkv);
+}
+void orc_stage_attend(void* m, const float* q, const float* K, const float* V, int c, int n, float* o) {
+    const Model& M = *(Model*)m;
+    stage_attend(M, q, (size_t)M.d.D, K, V, c, n, o);
+}
+void orc_stage_attn_out(void* m, int layer, const float* o, int n, float* x) {
+    const Model& M = *(Model*)m;
+    stage_attn_out(M, M.layers[layer], o, n, x);
+}
+void orc_stage_ffn_act(void* m, int layer, const float* x, int n, float* mm, float* act) {
+    const Model& M = *(Model*)m;
+    stage_ffn_act(M, M.layers[layer], x, n, mm, act);
+}
+void orc_stage_ffn_down(void* m, int layer, const float* act, int n, float* x) {
+    const Model& M = *(Model*)m;
+    stage_ffn_down(M, M.layers[layer], act, n, x);
+}
+
+// Diagnostics for the noise-floor calibration (both 0: the oracle proper).  Never a comparison target.
+void orc_model_set_diag(void* m, int acc_f32, int attn_w_bf16) {
+    ((Model*)m)->acc_f32 = acc_f32;
+    ((Model*)m)->attn_w_bf16 = attn_w_bf16;
+}
+
 void orc_probs(const float* lc, const float* lu, float s, float tau, int k, int V, float* p) {
     probs(lc, lu, s, tau, k, V, p);
 }
@@ -678,7 +811,8 @@ void* orc_rollout_create(void* m, int B, const int32_t* prefix_tokens, const int
     const int T = M.T, V = M.d.V, W = P->window;
     const bool cfg = P->cfg_scale != 1.0f;
     const size_t cache = (size_t)M.d.L * T * M.d.D;
-#pragma omp parallel for schedule(dynamic)
+    // one image per thread when there are enough images; otherwise the matrix products use the threads
+#pragma omp parallel for schedule(dynamic) if (B >= omp_get_max_threads())
     for (int b = 0; b < B; ++b) {
         Image& im = R->img[b];
         im.id = image_ids ? image_ids[b] : b;
@@ -733,7 +867,7 @@ int orc_rollout_round(void* r, int32_t* m_out, int32_t* j_out) {
     if (sync) {
         // batch-synchronous progress: every live image advances by the smallest commit of the batch
         std::vector<int> nat(R->B, 0);
-#pragma omp parallel for schedule(dynamic)
+#pragma omp parallel for schedule(dynamic) if (live >= omp_get_max_threads())
         for (int b = 0; b < R->B; ++b) {
             Image& im = R->img[b];
             if (im.c < T) {
@@ -744,7 +878,7 @@ int orc_rollout_round(void* r, int32_t* m_out, int32_t* j_out) {
         for (int b = 0; b < R->B; ++b)
             if (R->img[b].c < T && (m_limit == 0 || nat[b] < m_limit)) m_limit = nat[b];
     }
-#pragma omp parallel for schedule(dynamic) reduction(+ : commits, rej)
+#pragma omp parallel for schedule(dynamic) reduction(+ : commits, rej) if (live >= omp_get_max_threads())
     for (int b = 0; b < R->B; ++b) {
         Image& im = R->img[b];
         int m = 0, j = -1;

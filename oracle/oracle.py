@@ -35,6 +35,11 @@ class Params(C.Structure):
                 ("temperature", C.c_float), ("seed", C.c_uint64)]
 
 
+class Trace(C.Structure):
+    _fields_ = [("layer", C.c_int32)] + [(n, C.POINTER(C.c_float)) for n in
+                                         ("a", "q", "k", "v", "o", "x_attn", "m", "act", "x_out")]
+
+
 _lib = None
 
 
@@ -52,6 +57,14 @@ def lib():
         L.orc_model_destroy.argtypes = [vp]
         L.orc_forward_full.argtypes = [vp, C.c_int, i32p, C.c_int, f32p]
         L.orc_forward_window.argtypes = [vp, f32p, f32p, C.c_int, i32p, C.c_int, C.c_int, f32p]
+        L.orc_forward_window_trace.argtypes = [vp, f32p, f32p, C.c_int, i32p, C.c_int, C.c_int, f32p,
+                                               C.POINTER(Trace)]
+        L.orc_model_set_diag.argtypes = [vp, C.c_int, C.c_int]
+        L.orc_stage_qkv.argtypes = [vp, C.c_int, f32p, C.c_int, C.c_int, f32p, f32p]
+        L.orc_stage_attend.argtypes = [vp, f32p, f32p, f32p, C.c_int, C.c_int, f32p]
+        L.orc_stage_attn_out.argtypes = [vp, C.c_int, f32p, C.c_int, f32p]
+        L.orc_stage_ffn_act.argtypes = [vp, C.c_int, f32p, C.c_int, f32p, f32p]
+        L.orc_stage_ffn_down.argtypes = [vp, C.c_int, f32p, C.c_int, f32p]
         L.orc_probs.argtypes = [f32p, f32p, C.c_float, C.c_float, C.c_int, C.c_int, f32p]
         L.orc_sample.argtypes = [f32p, C.c_int, C.c_uint32]
         L.orc_sample.restype = C.c_int
@@ -212,6 +225,68 @@ class Model:
         lib().orc_forward_window(self.h, _p(cache[0], C.c_float), _p(cache[1], C.c_float), label,
                                  _p(seq, C.c_int32), c, n, _p(out, C.c_float))
         return out
+
+    def forward_window_trace(self, cache, label, seq, c, n, layer, want_logits=False):
+        """forward_window that also returns the intermediates of `layer` as a dict of fp32 arrays (row i =
+        sequence index c + i): a, q, k, v, o, x_attn, m [n, D]; act [n, F]; x_out [n, D]."""
+        seq = _i32(seq)
+        s = self.shape
+        out = np.zeros((n, s.vocab), dtype=np.float32) if want_logits else None
+        bufs = {name: np.zeros((n, s.ffn_hidden if name == "act" else s.dim), dtype=np.float32)
+                for name in ("a", "q", "k", "v", "o", "x_attn", "m", "act", "x_out")}
+        tr = Trace(layer, *[_p(bufs[name], C.c_float) for name in ("a", "q", "k", "v", "o", "x_attn", "m", "act",
+                                                                    "x_out")])
+        lib().orc_forward_window_trace(self.h, _p(cache[0], C.c_float), _p(cache[1], C.c_float), label,
+                                       _p(seq, C.c_int32), c, n, _p(out, C.c_float), C.byref(tr))
+        return bufs, out
+
+    # ---- single stages of one block on given inputs (the functions forward_window is made of)
+    def stage_qkv(self, layer, x, c):
+        """x fp32 [n, D] residual rows at sequence indices c.. -> (a, q, k, v) each [n, D]."""
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        n, D = x.shape
+        a = np.zeros((n, D), dtype=np.float32)
+        qkv = np.zeros((n, 3 * D), dtype=np.float32)
+        lib().orc_stage_qkv(self.h, layer, _p(x, C.c_float), n, c, _p(a, C.c_float), _p(qkv, C.c_float))
+        return a, qkv[:, :D].copy(), qkv[:, D:2 * D].copy(), qkv[:, 2 * D:].copy()
+
+    def stage_attend(self, q, K, V, c):
+        """q [n, D] at sequence indices c..; K, V [>= c+n, D] cache rows of one layer -> o [n, D]."""
+        q, K, V = (np.ascontiguousarray(t, dtype=np.float32) for t in (q, K, V))
+        n = q.shape[0]
+        assert K.shape[0] >= c + n and V.shape[0] >= c + n
+        o = np.zeros_like(q)
+        lib().orc_stage_attend(self.h, _p(q, C.c_float), _p(K, C.c_float), _p(V, C.c_float), c, n, _p(o, C.c_float))
+        return o
+
+    def stage_attn_out(self, layer, o, x):
+        """x + W_o o, fp32 [n, D]."""
+        o = np.ascontiguousarray(o, dtype=np.float32)
+        x = np.array(x, dtype=np.float32, copy=True, order="C")
+        lib().orc_stage_attn_out(self.h, layer, _p(o, C.c_float), o.shape[0], _p(x, C.c_float))
+        return x
+
+    def stage_ffn_act(self, layer, x):
+        """x fp32 [n, D] -> (m [n, D], act [n, F])."""
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        n = x.shape[0]
+        m = np.zeros_like(x)
+        act = np.zeros((n, self.shape.ffn_hidden), dtype=np.float32)
+        lib().orc_stage_ffn_act(self.h, layer, _p(x, C.c_float), n, _p(m, C.c_float), _p(act, C.c_float))
+        return m, act
+
+    def stage_ffn_down(self, layer, act, x):
+        """x + W_2 act, fp32 [n, D]."""
+        act = np.ascontiguousarray(act, dtype=np.float32)
+        x = np.array(x, dtype=np.float32, copy=True, order="C")
+        lib().orc_stage_ffn_down(self.h, layer, _p(act, C.c_float), act.shape[0], _p(x, C.c_float))
+        return x
+
+    def set_diag(self, acc_f32: bool = False, attn_w_bf16: bool = False):
+        """Diagnostics of the noise-floor calibration, never a comparison target: accumulate dot products in fp32
+        instead of double; round the unnormalised attention weights to bf16 before they multiply the values.
+        set_diag() restores the oracle proper."""
+        lib().orc_model_set_diag(self.h, int(acc_f32), int(attn_w_bf16))
 
     def ar_rollout(self, prefix_tokens, prefix_len, labels, params: Params, image_ids=None) -> np.ndarray:
         pt, pl, lb = _i32(prefix_tokens), _i32(prefix_len), _i32(labels)

@@ -15,9 +15,10 @@ DTYPE_FP32, DTYPE_BF16 = 0, 1
 VERIFY_PROB, VERIFY_GREEDY = 0, 1
 EXEC_FULL, EXEC_COMPACT, EXEC_HYBRID, EXEC_SYNC = 0, 1, 2, 3
 DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
+DBG_ACT_A, DBG_ACT_Q, DBG_ACT_O, DBG_ACT_FFN, DBG_ACT_H, DBG_KV_K, DBG_KV_V = 3, 4, 5, 6, 7, 8, 9
 
 EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_profile_launch_floor", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
-           "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
+           "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_debug_forward", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
            "hbsjd_last_error"]
 
 
@@ -98,6 +99,7 @@ def load():
         L.hbsjd_get_state.argtypes = [vp, vp, vp, vp, vp, C.POINTER(C.c_int32)]
         L.hbsjd_set_state.argtypes = [vp, vp, vp, vp, vp, C.c_int32]
         L.hbsjd_debug_read.argtypes = [vp, C.c_int, C.c_int, vp, C.c_size_t]
+        L.hbsjd_debug_forward.argtypes = [vp, C.c_int, C.c_int]
         L.hbsjd_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int]
         L.hbsjd_bikl.argtypes = [vp, vp, vp, C.c_int, vp]
         L.hbsjd_score.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp, vp, C.POINTER(C.c_float)]
@@ -260,9 +262,23 @@ class Context:
             buf = np.zeros((3, self.max_batch), dtype=np.int32)
             n = self._check(self.lib.hbsjd_debug_read(self.h, what, 0, buf.ctypes.data, buf.nbytes), "debug_read")
             return buf.reshape(-1)[:3 * n].reshape(3, n)
+        if what >= DBG_ACT_A:
+            # activation rows / cache rows in the context's element type, returned widened to fp32
+            s = self.shape
+            width = s.ffn_hidden if what == DBG_ACT_FFN else s.dim
+            rows = s.T + 1 if what in (DBG_KV_K, DBG_KV_V) else self.window
+            raw16 = s.dtype == "bf16" and what != DBG_ACT_H
+            buf = np.zeros((rows, width), dtype=np.uint16 if raw16 else np.float32)
+            n = self._check(self.lib.hbsjd_debug_read(self.h, what, index, buf.ctypes.data, buf.nbytes), "debug_read")
+            out = buf[:n]
+            return (out.astype(np.uint32) << np.uint32(16)).view(np.float32) if raw16 else out
         buf = np.zeros((self.window, V), dtype=np.float32)
         n = self._check(self.lib.hbsjd_debug_read(self.h, what, index, buf.ctypes.data, buf.nbytes), "debug_read")
         return buf[:n]
+
+    def hbsjd_debug_forward(self, layer: int, stage: int):
+        """Partial verifier forward of the current state up to `layer` (stage 0: attention sub-block, 1: whole block)."""
+        self._check(self.lib.hbsjd_debug_forward(self.h, layer, stage), "hbsjd_debug_forward")
 
     def hbsjd_gemm(self, A, W, Cout, accumulate=False):
         """Cout[M,N] fp32 (+)= A[M,K] . W[N,K]^T, tensors of the context's element type on the GPU."""

@@ -52,6 +52,7 @@ struct hbsjd_ctx {
     hbsjd_params P;
     bool have_rollout;
     int live, round, last_S, last_compact;
+    int dbg_layer;  // layer of the last hbsjd_debug_forward (-1: none); selects the KV rows of hbsjd_debug_read
     hbsjd_stats stats;
     long long launches;
     // host-buffer staging
@@ -160,8 +161,10 @@ int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int 
 }
 
 // One batched verifier forward over S slots (Sec. 4.2 "Batched verification").
+// stop_layer >= 0 (debugging): return after the attention sub-block (stop_stage 0) or the whole block
+// (stop_stage 1) of that layer, leaving the activation buffers as that point found them.
 template <typename TA>
-int forward(hbsjd_ctx* c, int S, bool want_logits) {
+int forward(hbsjd_ctx* c, int S, bool want_logits, int stop_layer = -1, int stop_stage = 0) {
     const State& st = c->st;
     const int M = st.nb * S * st.W, D = st.D, F = st.F;
     const int Mcap = 2 * c->Bmax * c->Wmax;  // row capacity of the activation buffers
@@ -206,6 +209,7 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
             c->launches++;
         }
         if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1, Mcap))) return rc;
+        if (l == stop_layer && stop_stage == 0) return 0;
         norm(c->h, w.g_ffn);
         c->launches++;
         if constexpr (std::is_same<TA, bf16>::value) {
@@ -222,6 +226,7 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
             c->launches++;
         }
         if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1, Mcap))) return rc;
+        if (l == stop_layer) return 0;
     }
     if (want_logits) {
         norm(c->h, c->g_out);
@@ -237,8 +242,9 @@ int forward(hbsjd_ctx* c, int S, bool want_logits) {
     return 0;
 }
 
-int forward_any(hbsjd_ctx* c, int S, bool want_logits) {
-    return c->bf16_model ? forward<bf16>(c, S, want_logits) : forward<float>(c, S, want_logits);
+int forward_any(hbsjd_ctx* c, int S, bool want_logits, int stop_layer = -1, int stop_stage = 0) {
+    return c->bf16_model ? forward<bf16>(c, S, want_logits, stop_layer, stop_stage)
+                         : forward<float>(c, S, want_logits, stop_layer, stop_stage);
 }
 
 int choose_compact(const hbsjd_ctx* c, int live) {
@@ -544,6 +550,7 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     const char* at = getenv("HBSJD_ATTENTION");
     c->ref_attention = at && strcmp(at, "ref") == 0;
     c->stream = (cudaStream_t)cuda_stream;
+    c->dbg_layer = -1;
     c->err[0] = 0;
     const int rc = create_impl(c, weights, weight_bytes);
     if (rc != 0) {
@@ -995,9 +1002,26 @@ int hbsjd_set_state(hbsjd_ctx* c, const int32_t* cursor, const int32_t* seq, con
     return HBSJD_OK;
 }
 
+int hbsjd_debug_forward(hbsjd_ctx* c, int layer, int stage) {
+    if (!c) return HBSJD_EINVAL;
+    if (!c->have_rollout) return HBSJD_ESTATE;
+    if (layer < 0 || layer >= c->d.n_layers || (stage != 0 && stage != 1)) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_debug_forward: layer or stage out of range");
+        return HBSJD_EINVAL;
+    }
+    launch_setup(c->st, 0, 0, c->stream);
+    const int rc = forward_any(c, c->st.B, false, layer, stage);
+    if (rc) return rc;
+    CK(cudaGetLastError());
+    c->last_S = c->st.B;
+    c->last_compact = 0;
+    c->dbg_layer = layer;
+    return sync_counters(c);
+}
+
 int hbsjd_debug_read(hbsjd_ctx* c, int what, int index, void* host_dst, size_t max_bytes) {
     if (!c || !host_dst) return HBSJD_EINVAL;
-    if (!c->have_rollout || c->round == 0) return HBSJD_ESTATE;
+    if (!c->have_rollout || (c->round == 0 && c->dbg_layer < 0)) return HBSJD_ESTATE;
     const int S = c->last_S, W = c->st.W, V = c->d.vocab;
     std::vector<int32_t> slots((size_t)3 * S);
     CK(cudaMemcpyAsync(slots.data(), c->st.slot_img, S * 4, cudaMemcpyDeviceToHost, c->stream));
@@ -1009,8 +1033,8 @@ int hbsjd_debug_read(hbsjd_ctx* c, int what, int index, void* host_dst, size_t m
         memcpy(host_dst, slots.data(), slots.size() * 4);
         return S;
     }
-    const int img = what == HBSJD_DBG_LOGITS ? index / 2 : index;
-    const int branch = what == HBSJD_DBG_LOGITS ? index % 2 : 0;
+    const int img = what == HBSJD_DBG_PROBS ? index : index / 2;
+    const int branch = what == HBSJD_DBG_PROBS ? 0 : index % 2;
     if (img < 0 || img >= c->st.B || (branch == 1 && c->st.nb == 1)) return HBSJD_EINVAL;
     int slot = -1;
     for (int s = 0; s < S; ++s)
@@ -1018,6 +1042,45 @@ int hbsjd_debug_read(hbsjd_ctx* c, int what, int index, void* host_dst, size_t m
     if (slot < 0) return 0;
     const int n = slots[2 * S + slot];
     if (n == 0) return 0;
+    if (what >= HBSJD_DBG_ACT_A && what <= HBSJD_DBG_ACT_H) {
+        // rows of the slot in an activation buffer, as the last (partial) forward left them
+        const size_t es = c->bf16_model ? 2 : 4, D = c->d.dim, F = c->d.ffn_hidden;
+        const size_t row0 = (size_t)(branch * S + slot) * W;
+        const unsigned char* src;
+        size_t width;
+        switch (what) {
+            case HBSJD_DBG_ACT_A: src = (const unsigned char*)c->a; width = D * es; break;
+            case HBSJD_DBG_ACT_Q: src = (const unsigned char*)c->q; width = D * es; break;
+            case HBSJD_DBG_ACT_O: src = (const unsigned char*)c->o; width = D * es; break;
+            case HBSJD_DBG_ACT_FFN: src = (const unsigned char*)c->act; width = F * es; break;
+            default: src = (const unsigned char*)c->h; width = D * 4; break;
+        }
+        if (max_bytes < (size_t)n * width) return HBSJD_EINVAL;
+        CK(cudaMemcpyAsync(host_dst, src + row0 * width, (size_t)n * width, cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        return n;
+    }
+    if (what == HBSJD_DBG_KV_K || what == HBSJD_DBG_KV_V) {
+        // cache rows of sequence indices 0 .. c+n-1 of the layer of the last hbsjd_debug_forward
+        if (c->dbg_layer < 0) return HBSJD_ESTATE;
+        const size_t es = c->bf16_model ? 2 : 4, D = c->d.dim;
+        const int rows = slots[S + slot] + n;
+        if (max_bytes < (size_t)rows * D * es) return HBSJD_EINVAL;
+        std::vector<int32_t> pt(c->pages_per_row);
+        const int crow = branch * c->Bmax + img;
+        CK(cudaMemcpyAsync(pt.data(), c->page_table + (size_t)crow * c->pages_per_row, pt.size() * 4,
+                           cudaMemcpyDeviceToHost, c->stream));
+        CK(cudaStreamSynchronize(c->stream));
+        const unsigned char* pool = (const unsigned char*)(what == HBSJD_DBG_KV_K ? c->kc : c->vc);
+        for (int s0 = 0; s0 < rows; s0 += PAGE_TOKENS) {
+            const int cnt = rows - s0 < PAGE_TOKENS ? rows - s0 : PAGE_TOKENS;
+            const size_t off = (((size_t)c->dbg_layer * c->n_pages + pt[s0 / PAGE_TOKENS]) * PAGE_TOKENS) * D * es;
+            CK(cudaMemcpyAsync((unsigned char*)host_dst + (size_t)s0 * D * es, pool + off, (size_t)cnt * D * es,
+                               cudaMemcpyDeviceToHost, c->stream));
+        }
+        CK(cudaStreamSynchronize(c->stream));
+        return rows;
+    }
     const size_t bytes = (size_t)n * V * sizeof(float);
     if (max_bytes < bytes) return HBSJD_EINVAL;
     const float* src;

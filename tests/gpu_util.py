@@ -42,6 +42,65 @@ def bf16_logit_tol(sigma, n_layers):
     return std, max(2e-2, 5.5 * std)
 
 
+def noise_floor(model, w, toks_row, label, c):
+    """Logit noise floor of bf16 activations at one window: the oracle against ITSELF in its diagnostic form --
+    every dot product accumulated in fp32 instead of double, and the attention weights rounded to bf16 before they
+    multiply the values (the tensor-core formulation of attention); nothing else changed -- on sequence indices
+    c .. c+n-1 after pre-filling 0 .. c-1.  A difference of one ulp anywhere flips bf16 roundings downstream,
+    after which the two runs differ at bf16-noise level; this measures how much of a logit that is at this
+    depth and logit scale: what two correct bf16 implementations must be expected to differ by.  The
+    diagnostic form is never a comparison target.  Returns (max |diff|, sum |diff|, number of logits, logit std)."""
+    T, W = w.shape.T, w.window
+    seq = np.zeros(T + 1, dtype=np.int32)
+    seq[1:] = toks_row
+    n = min(W, T - c)
+    out = []
+    for diag in (False, True):
+        model.set_diag(acc_f32=diag, attn_w_bf16=diag)
+        try:
+            cache = model.new_cache()
+            for pc in range(0, c, W):
+                model.forward_window(cache, label, seq, pc, min(W, c - pc), want_logits=False)
+            out.append(model.forward_window(cache, label, seq, c, n))
+        finally:
+            model.set_diag()
+    d = np.abs(out[0].astype(np.float64) - out[1].astype(np.float64))
+    return float(d.max()), float(d.sum()), int(d.size), float(out[0].std())
+
+
+def floor_of(model, w, toks, lab, k, ids):
+    """Noise floor over the first windows of the images `ids`: (max, mean over all their logits)."""
+    fl = [noise_floor(model, w, toks[b], int(lab[b]), int(k[b])) for b in ids if k[b] < w.shape.T]
+    return max(f[0] for f in fl), sum(f[1] for f in fl) / sum(f[2] for f in fl)
+
+
+def check_logits_against_floor(rep, floor_max, floor_mean, label="", max_factor=2.0, mean_factor=1.5):
+    """The GPU may differ from the oracle by what the oracle differs from its own diagnostic form (fp32 sums,
+    bf16 attention weights).  Measured: GPU error = 0.97-1.03 x the floor (maximum and mean) when the floor is
+    taken on every compared window (small models), 1.2 x the mean and up to 1.5 x the maximum when the floor is
+    sampled on the first windows only (full size: the GPU's maximum is then over 20-50 times more logits).  The
+    default factors fit the sampled case; callers with a per-window floor pass 1.3.  Prints both figures, so
+    that the measured ratio is on record in the test log."""
+    mean = rep["abs_err_sum"] / rep["abs_err_n"]
+    worst = max([min(x for x in (f.get("u_minus_alpha"), f.get("cdf_dist"), f.get("argmax_gap")) if x is not None)
+                 for f in rep["flips"]] or [0.0])
+    print(label, dict(gpu_max=round(rep["max_logit_err"], 4), gpu_mean=round(mean, 5), floor_max=round(floor_max, 4),
+                      floor_mean=round(floor_mean, 5), tokens=rep["tokens"], same=rep["same"],
+                      flips=len(rep["flips"]), widest_flip_margin=round(worst, 4), p_excess=rep["max_p_err"]))
+    assert rep["max_logit_err"] <= max_factor * floor_max, (rep["max_logit_err"], floor_max)
+    assert mean <= mean_factor * floor_mean, (mean, floor_mean)
+
+
+def check_flips_explained(rep):
+    """Every decision on which the GPU and the oracle differ must be reproduced bit for bit by the oracle's own
+    verification when it is fed the GPU's probabilities of that position (lockstep records this per flip), and
+    those probabilities must be the oracle's pipeline applied to the GPU's logits: the logit difference, bounded
+    separately against the noise floor, is then the only cause."""
+    assert rep["replay_mismatch"] == 0
+    for f in rep["flips"]:
+        assert f["replay_ok"] is True, f
+
+
 def residual_cdf_distance(p, q, is_delta, z, word):
     """Distance (as a fraction of the total mass) of the fixed-point target of `word` from the
     nearest bin edge of the replacement distribution."""
@@ -60,9 +119,13 @@ def residual_cdf_distance(p, q, is_delta, z, word):
 
 
 def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, max_rounds=None, gpu_batch=None,
-             check_replay=True):
+             check_replay=True, park_others=True, floor_every_round=False):
     """Runs the oracle and the GPU round by round, the GPU state re-synchronised to the oracle's before
-    each round.  `image_ids` restricts the oracle to a subset of the GPU batch.  Returns a report dict."""
+    each round.  `image_ids` restricts the oracle to a subset of the GPU batch; the other images are parked as
+    finished, or (park_others=False) keep rolling out on the GPU beside the followed ones, so that the forward
+    has the full batch's rows.  floor_every_round (small models): the noise floor (see noise_floor) is measured
+    on every window that is compared, by full recompute, so that the floor's maximum is taken over as many
+    logits as the GPU's; report keys floor_max / floor_sum / floor_n.  Returns a report dict."""
     ids = list(range(len(k))) if image_ids is None else list(image_ids)
     V, T, W = w.shape.vocab, w.shape.T, w.window
     P = orc_params(w, seed, greedy=greedy)
@@ -86,7 +149,8 @@ def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, ma
         cur[ids], seq[ids], dl[ids], qb[ids] = o_cur, o_seq, o_dl, o_qb
         # images outside the subset are parked as finished
         others = [b for b in range(len(k)) if b not in ids]
-        cur[others] = T
+        if park_others:
+            cur[others] = T
         ctx.hbsjd_set_state(o_r, cur, seq, dl, qb)
         ctx.hbsjd_round()
         g_r, g_cur, g_seq, g_dl, g_qb = ctx.hbsjd_get_state()
@@ -101,6 +165,18 @@ def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, ma
             n = min(W, T - c)
             gl = ctx.hbsjd_debug_read(binding.DBG_LOGITS, 2 * b)
             ol = orc.last_logits(x, 0)
+            if floor_every_round:
+                both = []
+                for diag in (False, True):
+                    model.set_diag(acc_f32=diag, attn_w_bf16=diag)
+                    try:
+                        both.append(model.forward_full(int(lab[b]), o_seq[x][:c + n])[c:].astype(np.float64))
+                    finally:
+                        model.set_diag()
+                d = np.abs(both[0] - both[1])
+                rep["floor_max"] = max(rep.get("floor_max", 0.0), float(d.max()))
+                rep["floor_sum"] = rep.get("floor_sum", 0.0) + float(d.sum())
+                rep["floor_n"] = rep.get("floor_n", 0) + d.size
             rep["max_logit_err"] = max(rep["max_logit_err"], float(np.abs(gl - ol).max()))
             rep["logit_std"] = max(rep["logit_std"], float(ol.std()))
             rep["abs_err_sum"] += float(np.abs(gl - ol).sum())
@@ -114,7 +190,8 @@ def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, ma
             # probabilities from the GPU's own logits through the oracle's pipeline
             pl = np.stack([O.probs(gl[i], glu[i] if w.cfg_scale != 1.0 else None, s=w.cfg_scale, tau=w.temperature,
                                    k=w.top_k) for i in range(n)])
-            rep["max_p_err"] = max(rep["max_p_err"], float((np.abs(gp_ - pl) - 1e-4 * pl).max()))
+            rep["max_p_err"] = max(rep["max_p_err"], float((np.abs(gp_ - pl) - 1e-5 * pl).max()))
+            ok = None
             if check_replay:
                 # verify / commit / refresh replayed by the oracle on the GPU's probabilities: bit-exact
                 s2, d2 = o_seq[x].copy(), o_dl[x].copy()
@@ -140,7 +217,9 @@ def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, ma
                 i = same  # window position whose decision differs
                 t = c + i + 1
                 words = O.philox([b, t, o_r, 0], [seed & 0xffffffff, seed >> 32])
-                info = dict(image=b, round=o_r, pos=t, m_gpu=m_g, m_orc=m_o)
+                # replay_ok: the oracle's own verification, fed the GPU's probabilities of this round, takes the
+                # GPU's decision bit for bit -- the flip comes from the logits alone
+                info = dict(image=b, round=o_r, pos=t, m_gpu=m_g, m_orc=m_o, replay_ok=ok)
                 if greedy:
                     # the GPU's argmax at this position is the token it committed there
                     if t <= c + m_g:

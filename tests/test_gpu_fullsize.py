@@ -3,9 +3,12 @@ rows, window 32 -> 8192 token rows per forward, the launch configuration bench.p
 configurations B (12 layers, no guidance), XL (36 layers, 24 x 24 tokens) and stress (L shape, batch 256, bimodal
 prefix lengths).
 
-The oracle needs up to half a minute per image-round at these sizes, so element-wise parity is taken on sampled
-outputs: one image (the one with the shortest prefix) is followed in lockstep for two rounds while the GPU runs
-the whole batch shape; everything else is checked through properties that hold at any size."""
+The oracle needs seconds per image-round at these sizes, so element-wise parity is taken on sampled outputs: three
+images per configuration (shortest, median, longest prefix) are followed in lockstep for four rounds, and one image
+of L to completion, while the GPU runs the whole batch shape; everything else is checked through properties that
+hold at any size.  The logit tolerance is not a formula: it is the oracle's own noise floor (the oracle against
+its diagnostic form: fp32 instead of double sums, attention weights rounded to bf16), measured in the same test on
+the first windows of the same images."""
 import numpy as np
 import pytest
 
@@ -57,18 +60,35 @@ def test_fullsize_properties(big):
     assert not np.array_equal(other.cpu().numpy(), ref)
 
 
-def test_fullsize_sampled_image_in_lockstep_with_the_oracle(big):
-    w, weights, ctx, toks, k, lab = big
-    b = int(np.argmin(k))  # shortest prefix: cheapest prefill for the oracle
-    model = O.Model(w.shape, weights)
-    rep = G.lockstep(ctx, model, w, toks, k, lab, 23, image_ids=[b], max_rounds=2)
-    std, tol = G.bf16_logit_tol(rep["logit_std"], w.shape.n_layers)
-    assert rep["max_logit_err"] <= tol, (rep["max_logit_err"], tol)
-    assert rep["abs_err_sum"] / rep["abs_err_n"] <= std, (rep["abs_err_sum"] / rep["abs_err_n"], std)
+def _check_against_floor(rep, model, w, toks, lab, k, ids, label):
+    floor_max, floor_mean = G.floor_of(model, w, toks, lab, k, ids)
+    G.check_logits_against_floor(rep, floor_max, floor_mean, label)
     assert rep["max_p_err"] <= 1e-6
-    assert rep["replay_mismatch"] == 0
-    assert rep["tokens"] >= 2
-    margin = float(np.expm1(2 * tol))
-    for f in rep["flips"]:
-        near = [x for x in (f.get("u_minus_alpha"), f.get("cdf_dist")) if x is not None]
-        assert near and min(near) < margin, f
+    G.check_flips_explained(rep)
+
+
+def test_fullsize_sampled_images_in_lockstep_with_the_oracle(big):
+    """Three images -- shortest, median and longest prefix -- followed for four rounds while the GPU runs the whole
+    batch shape: contexts of several pages, prefixes written by chunked pre-filling, cursors inside pages."""
+    w, weights, ctx, toks, k, lab = big
+    order = np.argsort(k, kind="stable")
+    ids = sorted({int(order[0]), int(order[len(order) // 2]), int(order[-1])})
+    model = O.Model(w.shape, weights)
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 23, image_ids=ids, max_rounds=4, park_others=False)
+    assert rep["tokens"] >= 4 * len(ids)
+    _check_against_floor(rep, model, w, toks, lab, k, ids, f"{w.name} ids {ids} k {[int(k[b]) for b in ids]}")
+
+
+def test_fullsize_one_image_to_completion(big):
+    """One image of workload L followed in lockstep until it is complete (40 tokens to generate), through the
+    ragged last windows n < W, with the rest of the batch live beside it on the GPU."""
+    w, weights, ctx, toks, k, lab = big
+    if w.name != "L":
+        pytest.skip("one configuration is enough for the run to completion")
+    k2 = k.copy()
+    b = 5
+    k2[b] = w.shape.T - 40
+    model = O.Model(w.shape, weights)
+    rep = G.lockstep(ctx, model, w, toks, k2, lab, 29, image_ids=[b], park_others=False)
+    assert rep["tokens"] == 40
+    _check_against_floor(rep, model, w, toks, lab, k2, [b], f"{w.name} image {b} to completion")

@@ -1,22 +1,23 @@
 """Parity of the CUDA rollout path (through the C ABI) with the CPU oracle.
 
 Tolerances:
-  forward logits      max-abs <= 1e-4 (fp32 model); bf16 model: <= max(2e-2, 5.5 s) with
-                      s = std(logits) (2^-9 / sqrt 3) sqrt(6 L + 1) (gpu_util.bf16_logit_tol): bf16 rounding
-                      of the activations is a RELATIVE error per rounding point that accumulates over the
-                      layers, so the absolute logit error grows with the logit scale and the depth; the mean
-                      absolute error must stay below s.  With a plain N(0, 0.02) head (logit std < 1) the
-                      literal bound 2e-2 holds and is asserted below; the benchmark's entropy-scaled heads
-                      have logit std 2.5-4.5.
-  probabilities       |p_gpu - p_oracle(gpu logits)| <= 1e-6 + 1e-4 p   (expf vs exp, fp32 sums)
+  forward logits      fp32 model: max-abs <= 1e-4.  bf16 model: bounded by the oracle's own NOISE FLOOR, measured in
+                      the test: the oracle against its diagnostic form, fp32 sums and bf16 attention weights (gpu_util.noise_floor).
+                      One ulp of difference in a sum flips bf16 roundings downstream, so any two correct
+                      implementations that accumulate differently differ by that much; the GPU must stay within
+                      1.3 times the floor's maximum and mean (measured 0.97-1.03), the floor taken on every
+                      compared window; full-size tests sample the floor and allow 2 x / 1.5 x.  With a plain N(0, 0.02) head (logit std
+                      < 1) the literal bound 2e-2 holds and is asserted; the benchmark's entropy-scaled heads have
+                      logit std 2.5-4.5 and a floor of 0.03-0.13.
+  probabilities       |p_gpu - p_oracle(gpu logits)| <= 1e-6 + 1e-5 p   (ex2.approx vs exp, fp32 sums)
   verify/commit/refresh, initial windows, compaction tables: bit-exact given the same p, q, words
-  end to end (lockstep): plain head: >= 99 % of committed tokens identical and every differing decision
-                      within 1e-3 of its threshold.  Entropy-scaled bf16 head: >= 95 % identical and every
-                      differing decision explained by the logit tolerance t: |u - alpha| <= e^{2t} - 1,
-                      sampling target within e^{2t} - 1 (as a probability mass) of a bin edge, or (greedy) the
-                      two argmax candidates within a factor e^{2t}.  A near-uniform distribution over k kept
-                      tokens has k thresholds per decision, each moved by the relative error of p, so the
-                      flip rate grows with both the logit error and the entropy; 99 % needs fp32 activations."""
+  end to end (lockstep): fp32 and plain head: >= 99 % of committed tokens identical and every differing decision
+                      within 1e-3 of its threshold.  Entropy-scaled bf16 head: the identical fraction is 93-98 %
+                      (a distribution over k kept tokens has k sampling thresholds per decision, each moved by the
+                      relative error of p: 99 % needs fp32 activations) -- asserted as a regression floor; every
+                      differing decision must be EXPLAINED: the oracle's verification fed the GPU's probabilities
+                      of that position reproduces the GPU's decision bit for bit (gpu_util.check_flips_explained),
+                      so the logit difference, bounded above, is its only cause."""
 import numpy as np
 import pytest
 
@@ -30,6 +31,15 @@ pytestmark = pytest.mark.gpu
 def _ctx(w, max_batch=None, max_window=None, weights=None):
     return binding.Context(w.shape, G.weights_for(w) if weights is None else weights, max_batch or w.batch,
                            max_window or w.window)
+
+
+def _check_bf16(rep, model, w, toks, k, lab, min_same, label):
+    """bf16 model: logits against the measured noise floor, probabilities, bit-exact replays, explained flips."""
+    floor_max, floor_mean = rep["floor_max"], rep["floor_sum"] / rep["floor_n"]  # lockstep(floor_every_round=True)
+    G.check_logits_against_floor(rep, floor_max, floor_mean, label, max_factor=1.3, mean_factor=1.3)
+    assert rep["max_p_err"] <= 1e-6, rep["max_p_err"]
+    assert rep["tokens"] > 0 and rep["same"] >= min_same * rep["tokens"], (rep["same"], rep["tokens"])
+    G.check_flips_explained(rep)
 
 
 def _check_report(rep, logit_tol, min_same=0.99, margin=1e-3):
@@ -85,10 +95,8 @@ def test_tiny_bf16_cfg_topk_lockstep(greedy):
     k[0], k[1] = 0, w.shape.T - 3  # an empty prefix and a nearly complete one (ragged tail: n < W)
     model = O.Model(w.shape, G.weights_for(w))
     ctx = _ctx(w)
-    rep = G.lockstep(ctx, model, w, toks, k, lab, 11, greedy=greedy)
-    std, tol = G.bf16_logit_tol(rep["logit_std"], w.shape.n_layers)
-    assert rep["abs_err_sum"] / rep["abs_err_n"] <= std
-    _check_report(rep, tol, min_same=0.95, margin=float(np.expm1(2 * tol)))
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 11, greedy=greedy, floor_every_round=True)
+    _check_bf16(rep, model, w, toks, k, lab, 0.95, f"tiny_bf16 greedy={greedy}")
     ctx.hbsjd_destroy()
 
 
@@ -117,10 +125,8 @@ def test_small_bf16_wide_windows_multi_page(W):
     k[0], k[1] = 0, w.shape.T - 5
     model = O.Model(w.shape, G.weights_for(w))
     ctx = _ctx(w)
-    rep = G.lockstep(ctx, model, w, toks, k, lab, 21, max_rounds=6)
-    std, tol = G.bf16_logit_tol(rep["logit_std"], w.shape.n_layers)
-    assert rep["abs_err_sum"] / rep["abs_err_n"] <= std
-    _check_report(rep, tol, min_same=0.93, margin=float(np.expm1(2 * tol)))
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 21, max_rounds=6, floor_every_round=True)
+    _check_bf16(rep, model, w, toks, k, lab, 0.93, f"small_bf16 W={W}")
     ctx.hbsjd_destroy()
 
 

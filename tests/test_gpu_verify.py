@@ -45,7 +45,7 @@ def test_verify_step_is_bit_exact_against_the_oracle(ctx, greedy, branches, top_
         for i in range(n):
             ref = O.probs(case["logits"][0, b, i], case["logits"][1, b, i] if branches == 2 else None,
                           s=case["cfg_scale"], k=top_k)
-            assert np.all(np.abs(p[b, i] - ref) <= 1e-6 + 1e-4 * ref)
+            assert np.all(np.abs(p[b, i] - ref) <= 1e-6 + 1e-5 * ref)
         # decision replayed on the GPU's probabilities
         s2, d2 = case["seq"][b].copy(), case["delta"][b].copy()
         nc, mm, jj = O.replay_round(V, T, W, H, greedy, seed, b, rnd, c, s2, d2, p[b, :n], case["q"][b],
