@@ -33,24 +33,37 @@ def _rope_factors(shape, n):
     return torch.polar(torch.ones_like(ang), ang)  # e^{i ang}
 
 
-def forward(shape, P, label, seq):
-    """seq: int array [n], seq[0] ignored.  Returns fp64 logits [n, V] (no bf16 rounding)."""
+BF16_POINTS = ("norm", "q", "k", "v", "o", "act")
+
+
+def _bf16(t):
+    """double -> float -> bfloat16 (round to nearest even) -> double, with torch's own casts."""
+    return t.to(torch.float32).to(torch.bfloat16).to(torch.float64)
+
+
+def forward(shape, P, label, seq, bf16_points=()):
+    """seq: int array [n], seq[0] ignored.  Returns fp64 logits [n, V].  bf16_points: the activations that are
+    rounded to bf16 -- any of "norm" (every RMSNorm output), "q", "k" (after the rotation), "v", "o" (attention
+    output), "act" (SwiGLU output); extra names "resid" (the residual stream) and "gu" (gate / up pre-activations)
+    exist so that a test can show that rounding at a point that is NOT on the list is detected."""
+    r = lambda name, t: _bf16(t) if name in bf16_points else t
     n = len(seq)
     Hh, dh, D = shape.n_heads, shape.head_dim, shape.dim
     x = torch.cat([P["cls"][label][None, :], P["tok"][torch.as_tensor(np.asarray(seq[1:], dtype=np.int64))]], 0)
     rot = _rope_factors(shape, n)[:, None, :]  # [n,1,dh/2]
     mask = torch.full((n, n), float("-inf"), dtype=torch.float64).triu(1)
     for Ly in P["layers"]:
-        a = _norm(x, Ly["g_attn"], shape.rms_eps)
+        a = r("norm", _norm(x, Ly["g_attn"], shape.rms_eps))
         qkv = a @ Ly["qkv"].T
         q, k, v = [t.reshape(n, Hh, dh) for t in qkv.split(D, dim=1)]
         qc = torch.view_as_real(torch.view_as_complex(q.reshape(n, Hh, dh // 2, 2).contiguous()) * rot).reshape(n, Hh, dh)
         kc = torch.view_as_real(torch.view_as_complex(k.reshape(n, Hh, dh // 2, 2).contiguous()) * rot).reshape(n, Hh, dh)
+        qc, kc, v = r("q", qc), r("k", kc), r("v", v)
         sc = torch.einsum("ihd,jhd->hij", qc, kc) / np.sqrt(dh) + mask[None]
-        o = torch.einsum("hij,jhd->ihd", torch.softmax(sc, -1), v).reshape(n, D)
-        x = x + o @ Ly["o"].T
-        m = _norm(x, Ly["g_ffn"], shape.rms_eps)
-        gu = m @ Ly["w13"].T
+        o = r("o", torch.einsum("hij,jhd->ihd", torch.softmax(sc, -1), v).reshape(n, D))
+        x = r("resid", x + o @ Ly["o"].T)
+        m = r("norm", _norm(x, Ly["g_ffn"], shape.rms_eps))
+        gu = r("gu", m @ Ly["w13"].T)
         F = shape.ffn_hidden
-        x = x + (torch.nn.functional.silu(gu[:, :F]) * gu[:, F:]) @ Ly["w2"].T
-    return (_norm(x, P["g_out"], shape.rms_eps) @ P["head"].T).numpy()
+        x = r("resid", x + r("act", torch.nn.functional.silu(gu[:, :F]) * gu[:, F:]) @ Ly["w2"].T)
+    return (r("norm", _norm(x, P["g_out"], shape.rms_eps)) @ P["head"].T).numpy()
