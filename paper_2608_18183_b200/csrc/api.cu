@@ -265,8 +265,15 @@ int sync_counters(hbsjd_ctx* c) {
         prof_resolve(c, nb * (keys * 2.0 * D * es + n * 2.0 * D * es), n * (nb + 1.0) * V * 4.0);
     }
     if (c->h_counters[CNT_ERROR] != 0) {
-        snprintf(c->err, sizeof(c->err), "a bounded device-side wait gave up (code %d)", c->h_counters[CNT_ERROR]);
+        const int code = c->h_counters[CNT_ERROR];
         cudaMemsetAsync(c->st.counters + CNT_ERROR, 0, sizeof(int32_t), c->stream);
+        if (code >= 16) {  // a kernel met rollout state that cannot be valid; it skipped the access
+            snprintf(c->err, sizeof(c->err), "invalid rollout state on the device (code %d: %s)", code,
+                     code == 16 ? "cursor out of range" : code == 17 ? "draft token out of range"
+                                                                     : "proposal row out of range");
+            return HBSJD_EINVAL;
+        }
+        snprintf(c->err, sizeof(c->err), "a bounded device-side wait gave up (code %d)", code);
         return HBSJD_ETIMEOUT;
     }
     return 0;
@@ -714,7 +721,7 @@ int hbsjd_verify(hbsjd_ctx* c, const hbsjd_verify_desc* d, const float* logits, 
     if (!d || !logits || !q_prev || !p_out || !cursor || !seq || !delta || !qbase || !m_out || d->batch < 1 ||
         d->batch > c->Bmax || d->window < 1 || d->window > c->Wmax || d->T < 1 || d->V < 4 || d->V % 4 ||
         d->V > 32768 || (d->branches != 1 && d->branches != 2) || d->history_offset < 1 ||
-        !(d->temperature > 0.f) || d->top_k < 0) {
+        !(d->temperature > 0.f) || !std::isfinite(d->temperature) || !std::isfinite(d->cfg_scale) || d->top_k < 0) {
         snprintf(c->err, sizeof(c->err), "hbsjd_verify: argument out of range");
         return HBSJD_EINVAL;
     }
@@ -723,7 +730,15 @@ int hbsjd_verify(hbsjd_ctx* c, const hbsjd_verify_desc* d, const float* logits, 
     memcpy(&vd, d, sizeof(vd));
     const VerifyScratch sc = verify_scratch_carve(c->verify_scratch, d->batch, d->window);
     CK(verify_enqueue(vd, sc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out, c->stream));
+    // the kernels check the caller's state arrays as they read them (cursor, draft tokens, proposal rows): a
+    // value that cannot be valid is recorded, its access skipped, and reported here
+    int32_t code = 0;
+    CK(cudaMemcpyAsync(&code, sc.counters + CNT_ERROR, sizeof(code), cudaMemcpyDeviceToHost, c->stream));
     CK(cudaStreamSynchronize(c->stream));
+    if (code != 0) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_verify: invalid state array on the device (code %d)", code);
+        return code >= 16 ? HBSJD_EINVAL : HBSJD_ETIMEOUT;
+    }
     return HBSJD_OK;
 }
 
@@ -988,6 +1003,12 @@ int hbsjd_set_state(hbsjd_ctx* c, const int32_t* cursor, const int32_t* seq, con
         for (size_t t = 1; t < T1; ++t)
             if (seq[b * T1 + t] < 0 || seq[b * T1 + t] >= c->d.vocab) {
                 snprintf(c->err, sizeof(c->err), "set_state: image %zu token %zu out of range", b, t);
+                return HBSJD_EINVAL;
+            }
+        // a sampled draft (delta = 0) at position t reads row t - qbase - 1 of the previous round's probabilities
+        for (int t = cursor[b] + 1; t < cursor[b] + c->st.W && t < c->T; ++t)
+            if (!delta[b * T1 + t] && t - qbase[b] - 1 >= c->Wmax) {
+                snprintf(c->err, sizeof(c->err), "set_state: image %zu draft %d has no proposal row", b, t);
                 return HBSJD_EINVAL;
             }
         live += cursor[b] < c->T;

@@ -101,6 +101,11 @@ void launch_commit(const State& st, const AcceptArgs& a, cudaStream_t s);
 // smallest commit over the live slots of this round, from the accept flags (batch-synchronous progress)
 void launch_sync_min(const State& st, const AcceptArgs& a, int32_t* m_sync, cudaStream_t s);
 int accept_smem_bytes(int V);
+// persistent form of launch_prob_accept for vocabularies up to 16384 (accept_persistent.cu)
+bool accept_persistent_supported(const State& st);
+void launch_accept_persistent(const State& st, const AcceptArgs& a, int n_sms, cudaStream_t s);
+// streaming multiprocessors of the current device
+int device_sm_count();
 void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_scale, float temperature, int top_k,
                   float* p, cudaStream_t s);
 

@@ -21,6 +21,10 @@ __global__ void k_setup(State st, int phase, int compact) {
         if (b < st.B) {
             if (phase == 0) {
                 c = st.cursor[b];
+                if (c < 0 || c > st.T) {  // cannot be valid: record it and leave the image out of the round
+                    atomicExch(&st.counters[CNT_ERROR], 16);
+                    c = st.T;
+                }
                 n = c < st.T ? min(st.W, st.T - c) : 0;
             } else {
                 c = st.pfill[b];

@@ -4,6 +4,7 @@
 #include <mutex>
 
 #include "../../include/hbsjd.h"
+#include "accept_common.cuh"
 #include "internal.h"
 
 namespace hbsjd {
@@ -130,9 +131,7 @@ void launch_calib_state(const State& st, int live, cudaStream_t s) {
 constexpr int ACC_THREADS = 512;
 constexpr int ACC_WARPS = ACC_THREADS / 32;
 
-// Work area + reduction scratch behind the V floats.  Sized so that three CTAs fit one SM at V = 16384.
-constexpr int SEL_BINS = 1024;
-constexpr int SEL_CAP = 1536;
+// Work area + reduction scratch behind the V floats.
 struct AccShared {
     unsigned int work[SEL_BINS + SEL_CAP];  // selection histogram, then the keys of the selected bin
     float redf[ACC_WARPS];
@@ -143,11 +142,6 @@ struct AccShared {
     uint32_t words[4];
     int jfirst;
 };
-
-__device__ __forceinline__ unsigned int float_key(float x) {
-    const unsigned int u = __float_as_uint(x);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
 
 __device__ __forceinline__ float block_max(float v, AccShared& sh) {
     v = warp_max(v);
@@ -171,16 +165,8 @@ __device__ __forceinline__ float block_sum(float v, AccShared& sh) {
     return r;
 }
 
-__device__ __forceinline__ unsigned int fixed_weight(float a) { return __float2uint_rd(a * 1073741824.0f); }
-
 // Warp w owns the contiguous segment [w * seg, (w+1) * seg) of the vocabulary (seg a multiple of 128).
 __device__ __forceinline__ int warp_segment(int V) { return (((V + ACC_WARPS - 1) / ACC_WARPS) + 127) / 128 * 128; }
-
-__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
-}
 
 // Fixed-point categorical pick over a[0..V) (shared memory) whose per-warp weight sums are in sh.redu
 // (all threads call; ends with a barrier).  Integer running sums: the result is the smallest v whose
@@ -493,11 +479,7 @@ __device__ void prob_pipeline(float* g, const float* __restrict__ lc, const floa
         // the count and costs a second pass if it was too high.
         const float mean = s1 / (float)V;
         const float sd = sqrtf(fmaxf(s2 / (float)V - mean * mean, 0.f));
-        const float f = fminf(0.5f, (1.5f * (float)top_k + 16.f) / (float)V);
-        const float tq = sqrtf(-2.0f * __logf(f));
-        const float zq = tq - (2.515517f + tq * (0.802853f + tq * 0.010328f)) /
-                                  (1.0f + tq * (1.432788f + tq * (0.189269f + tq * 0.001308f)));
-        theta = topk_threshold(g, V, (unsigned int)top_k, mn, mx, mean + zq * sd, sh);
+        theta = topk_threshold(g, V, (unsigned int)top_k, mn, mx, topk_guess(mean, sd, top_k, V), sh);
     } else {
         mx = block_max(mx, sh);  // the barriers inside also publish g
     }
@@ -505,8 +487,7 @@ __device__ void prob_pipeline(float* g, const float* __restrict__ lc, const floa
     // float compare; ex2.approx (relative error about 1e-6 over the range used) and a multiplication by
     // 1/sum replace expf and the division: both sit well inside the probability tolerance, and every
     // downstream decision uses these very numbers.
-    const float thr = theta == 0u ? -INFINITY
-                                  : __uint_as_float((theta & 0x80000000u) ? (theta & 0x7FFFFFFFu) : ~theta);
+    const float thr = theta == 0u ? -INFINITY : key_float(theta);
     float part = 0.f;
     for (int v = tid * 4; v < V; v += ACC_THREADS * 4) {
         float4 x = *reinterpret_cast<float4*>(g + v);
@@ -572,9 +553,21 @@ __global__ void __launch_bounds__(ACC_THREADS, 2) k_prob_accept(State st, Accept
 
     const size_t oidx = (size_t)img * st.Wmax + i;
     const bool last = (i == n - 1);
-    const int z = last ? 0 : st.seq[(size_t)img * (st.T + 1) + t];
+    int z = last ? 0 : st.seq[(size_t)img * (st.T + 1) + t];
     const bool is_delta = last ? false : (st.delta[(size_t)img * (st.T + 1) + t] != 0);
-    const int qi = (last || is_delta) ? 0 : (t - st.qbase[img] - 1);  // row of the previous round's probabilities
+    int qi = (last || is_delta) ? 0 : (t - st.qbase[img] - 1);  // row of the previous round's probabilities
+    // state that cannot be valid: record it, skip the access, treat the draft as rejected
+    bool bad = false;
+    if (z < 0 || z >= V) {
+        if (tid == 0) atomicExch(&st.counters[CNT_ERROR], ERR_BAD_TOKEN);
+        z = 0;
+        bad = true;
+    }
+    if (qi < 0 || qi >= st.Wmax) {
+        if (tid == 0) atomicExch(&st.counters[CNT_ERROR], ERR_BAD_PROPOSAL_ROW);
+        qi = 0;
+        bad = true;
+    }
     const float* qrow = a.pprev + ((size_t)img * st.Wmax + qi) * V;
 
     if (a.greedy) {
@@ -599,7 +592,7 @@ __global__ void __launch_bounds__(ACC_THREADS, 2) k_prob_accept(State st, Accept
             const int am = (int)(0xFFFFFFFFu - (unsigned)(b2 & 0xFFFFFFFFull));
             a.cand_rep[oidx] = am;
             a.cand_ref[oidx] = am;
-            a.flag[oidx] = (!last && z == am) ? 1 : 0;
+            a.flag[oidx] = (!last && !bad && z == am) ? 1 : 0;
         }
         return;
     }
@@ -612,7 +605,7 @@ __global__ void __launch_bounds__(ACC_THREADS, 2) k_prob_accept(State st, Accept
             if (is_delta) alpha = pz;
             else alpha = fminf(1.0f, __fdiv_rn(pz, qrow[z]));
             const float u = (float)(sh.words[0] >> 8) * (1.0f / 16777216.0f);
-            a.flag[oidx] = (u < alpha) ? 1 : 0;
+            a.flag[oidx] = (!bad && u < alpha) ? 1 : 0;
         }
     }
 
@@ -632,7 +625,23 @@ void launch_probs(const float* lc, const float* lu, int rows, int V, float cfg_s
     launch_k(k_probs, dim3(rows), dim3(ACC_THREADS), bytes, s, lc, lu, V, cfg_scale, temperature, top_k, p);
 }
 
+int device_sm_count() {
+    static int n[64] = {0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    if (!n[dev]) {
+        cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev);
+        if (n[dev] <= 0) n[dev] = 148;
+    }
+    return n[dev];
+}
+
 void launch_prob_accept(const State& st, const AcceptArgs& a, cudaStream_t s) {
+    if (accept_persistent_supported(st)) {
+        launch_accept_persistent(st, a, device_sm_count(), s);
+        return;
+    }
     static int configured[64] = {0};
     const int bytes = accept_smem_bytes(st.V);
     ensure_dynamic_smem(k_prob_accept, bytes, configured);
@@ -698,9 +707,13 @@ __global__ void __launch_bounds__(ACC_THREADS) k_commit(State st, AcceptArgs a) 
         const float* prow = a.pcur + ((size_t)img * st.Wmax + is) * V;
         const bool reject = j >= 0;
         const int z = reject ? seq[t] : -1;
-        const bool is_delta = reject && dl[t] != 0;
-        const float* qrow =
-            (reject && !is_delta) ? a.pprev + ((size_t)img * st.Wmax + (t - st.qbase[img] - 1)) * V : nullptr;
+        bool is_delta = reject && dl[t] != 0;
+        int qi = t - st.qbase[img] - 1;
+        if (reject && !is_delta && (qi < 0 || qi >= st.Wmax)) {  // cannot be valid: record it, skip the access
+            if (tid == 0) atomicExch(&st.counters[CNT_ERROR], ERR_BAD_PROPOSAL_ROW);
+            is_delta = true;
+        }
+        const float* qrow = (reject && !is_delta) ? a.pprev + ((size_t)img * st.Wmax + qi) * V : nullptr;
         const int seg = warp_segment(V);
         const int vend = min(V, (wid + 1) * seg);
         for (int pass = 0; pass < 2; ++pass) {
@@ -909,7 +922,8 @@ extern "C" int hbsjd_verify_static(void* cuda_stream, const hbsjd_verify_desc* d
     if (!d || !logits || !q_prev || !p_out || !cursor || !seq || !delta || !qbase || !m_out) return HBSJD_EINVAL;
     if (d->batch < 1 || d->batch > 1024 || d->window < 1 || d->window > 64 ||
         (long)d->batch * d->window > 16384 || d->T < 1 || d->V < 4 || d->V % 4 || d->V > 32768 ||
-        (d->branches != 1 && d->branches != 2) || d->history_offset < 1 || !(d->temperature > 0.f) || d->top_k < 0)
+        (d->branches != 1 && d->branches != 2) || d->history_offset < 1 || !(d->temperature > 0.f) ||
+        !(d->temperature < INFINITY) || !(fabsf(d->cfg_scale) < INFINITY) || d->top_k < 0)
         return HBSJD_EINVAL;
     if (verify_scratch_bytes(d->batch, d->window) > kStaticScratchBytes) return HBSJD_EINVAL;
     int dev = 0;
@@ -934,6 +948,11 @@ extern "C" int hbsjd_verify_static(void* cuda_stream, const hbsjd_verify_desc* d
     // every (image, position) that is read back, so stale contents of the previous call are never used
     if (verify_enqueue(vd, sc, logits, q_prev, p_out, cursor, seq, delta, qbase, m_out, s) != cudaSuccess)
         return HBSJD_ECUDA;
+    // the kernels record state that cannot be valid (and skip the access): read the record back (no allocation)
+    int32_t code = 0;
+    if (cudaMemcpyAsync(&code, sc.counters + CNT_ERROR, sizeof(code), cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return HBSJD_ECUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return HBSJD_ECUDA;
+    if (code != 0) return code >= 16 ? HBSJD_EINVAL : HBSJD_ETIMEOUT;
     return HBSJD_OK;
 }

@@ -73,3 +73,50 @@ def test_verify_rejects_bad_arguments(ctx):
         with pytest.raises(binding.HbsjdError) as e:
             ctx.hbsjd_verify(desc, d["logits"], d["q"], p_out, d["cursor"], d["seq"], d["delta"], d["qbase"], m_out)
         assert e.value.code == -1
+
+
+@pytest.mark.parametrize("what", ["token_high", "token_negative", "cursor_negative", "cursor_high", "qbase", "cfg_nan"])
+def test_verify_reports_invalid_state_arrays_instead_of_touching_memory(ctx, what):
+    """The state arrays of hbsjd_verify live on the device and cannot be checked on the host before the launch:
+    the kernels bound every index they derive from them.  A draft token outside the vocabulary, a cursor outside
+    0..T or a proposal row outside the window is recorded, its access skipped, and the call returns
+    HBSJD_EINVAL; the context stays usable."""
+    import torch
+    case = G.verify_case(5, B=8, W=8, T=32, V=256)
+    b = 4
+    c = int(case["cursor"][b])
+    assert c + 2 < case["T"]
+    case["delta"][b, c + 1] = 0  # a sampled draft: its proposal row is read
+    if what == "token_high":
+        case["seq"][b, c + 1] = case["V"] + 5
+    elif what == "token_negative":
+        case["seq"][b, c + 1] = -3
+    elif what == "cursor_negative":
+        case["cursor"][b] = -2
+    elif what == "cursor_high":
+        case["cursor"][b] = case["T"] + 7
+    elif what == "qbase":
+        case["qbase"][b] = c - 200  # row t - qbase - 1 far outside the window
+    desc = G.verify_desc(case, 1, 0)
+    if what == "cfg_nan":
+        desc.cfg_scale = float("nan")
+    d = {k: G.dev(case[k]) for k in ("logits", "q", "cursor", "seq", "delta", "qbase")}
+    p_out = torch.zeros((8, 8, 256), device="cuda")
+    m_out = torch.zeros(8, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream()
+    for call in (lambda: ctx.hbsjd_verify(desc, d["logits"], d["q"], p_out, d["cursor"], d["seq"], d["delta"],
+                                          d["qbase"], m_out),
+                 lambda: binding.hbsjd_verify_static(stream, desc, d["logits"], d["q"], p_out, d["cursor"], d["seq"],
+                                                     d["delta"], d["qbase"], m_out)):
+        for k in ("cursor", "seq", "delta", "qbase"):
+            d[k].copy_(G.dev(case[k]))
+        with pytest.raises(binding.HbsjdError) as e:
+            call()
+        assert e.value.code == -1
+    torch.cuda.synchronize()
+    # a valid call right after succeeds
+    good = G.verify_case(6, B=8, W=8, T=32, V=256)
+    dg = {k: G.dev(good[k]) for k in ("logits", "q", "cursor", "seq", "delta", "qbase")}
+    ctx.hbsjd_verify(G.verify_desc(good, 1, 0), dg["logits"], dg["q"], p_out, dg["cursor"], dg["seq"], dg["delta"],
+                     dg["qbase"], m_out)
+    assert int(m_out.cpu().numpy()[good["cursor"] < good["T"]].min()) >= 1
