@@ -5,6 +5,7 @@
     python microbench.py gemm     # decoder GEMM shapes of a workload, each timed alone
     python microbench.py bikl     # bidirectional-KL reduction (Eq. 3) on 4096 row pairs
     python microbench.py score    # teacher/student scoring of a batch of trajectories (Eq. 3)
+    python microbench.py attention  # ragged attention at fixed context lengths (--workload L|XL, --contexts a,b,..)
 
 The rollouts of bench.py run random-weight models whose acceptance pattern is not the paper's; `accept` feeds
 the verification kernels synthetic (p, q) pairs instead: targets p = softmax(l), proposals q = softmax(l + sigma *
@@ -254,9 +255,43 @@ def bench_score(args):
     tea.hbsjd_destroy()
 
 
+def bench_attention(args):
+    """The ragged attention kernel at fixed context lengths: every image of the workload's batch gets the same
+    prefix, the prefix is pre-filled, then the verifier forward runs once under the library's per-class event
+    timing.  Bytes: K and V rows 0..c+n-1 read per physical row, q read and output written per input."""
+    import torch
+    from paper_2608_18183_b200 import binding, synth
+    w = synth.WORKLOADS[args.workload]
+    s = w.shape
+    B = args.batch or w.batch
+    ctx = binding.Context(s, synth.make_weights(s, w.weight_seed), B, w.window)
+    toks, _, lab = synth.make_inputs(w, batch=B)
+    floor_us = ctx.hbsjd_profile_launch_floor(200)
+    for c in [int(x) for x in args.contexts.split(",")]:
+        k = np.full(B, min(c, s.T - 1), dtype=np.int32)
+        p = binding.make_params(w.window, w.history_offset, w.cfg_scale, w.temperature, w.top_k, binding.VERIFY_PROB,
+                                binding.EXEC_FULL, 0, 1, 0)
+        ctx.hbsjd_rollout(torch.from_numpy(toks).cuda(), torch.from_numpy(k).cuda(), torch.from_numpy(lab).cuda(), p)
+        ctx.hbsjd_debug_forward(s.n_layers - 1, 0)  # warm
+        ctx.hbsjd_profile(True)
+        for _ in range(3):
+            ctx.hbsjd_debug_forward(s.n_layers - 1, 0)
+        pr = ctx.hbsjd_profile_read()["attention"]
+        ctx.hbsjd_profile(False)
+        us = pr["ms"] * 1e3 / pr["launches"]
+        alg = pr["work"] / pr["launches"]
+        print(json.dumps({"case": "attention", "workload": args.workload, "batch": B, "window": w.window,
+                          "context": int(k[0]), "us_per_launch": round(us, 2), "launches": pr["launches"],
+                          "algorithmic_bytes": alg, "GB_s": round(alg / us / 1e3, 1),
+                          "GB_s_net_of_launch_floor": round(alg / (us - floor_us) / 1e3, 1),
+                          "event_pair_launch_floor_us": round(floor_us, 2)}))
+    ctx.hbsjd_destroy()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
-    ap.add_argument("case", choices=["accept", "probs", "gemm", "bikl", "score"])
+    ap.add_argument("case", choices=["accept", "probs", "gemm", "bikl", "score", "attention"])
+    ap.add_argument("--contexts", default="0,32,64,128,192,223")
     ap.add_argument("--workload", default="L")
     ap.add_argument("--batch", type=int, default=0)
     ap.add_argument("--window", type=int, default=32)
@@ -270,7 +305,7 @@ def main(argv=None):
     if args.case in ("probs", "bikl") and not args.rows:
         args.rows = 4096
     {"accept": bench_accept, "probs": bench_probs, "gemm": bench_gemm, "bikl": bench_bikl,
-     "score": bench_score}[args.case](args)
+     "score": bench_score, "attention": bench_attention}[args.case](args)
 
 
 if __name__ == "__main__":

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIBDIR = os.path.join(HERE, "lib")
 LIB = os.path.join(LIBDIR, "libhbsjd.so")
-SOURCES = ["api.cu", "model_kernels.cu", "state_kernels.cu", "gemm_tcgen05.cu", "attention_mma.cu", "score_kernels.cu",
+SOURCES = ["api.cu", "model_kernels.cu", "state_kernels.cu", "gemm_tcgen05.cu", "attention_tma.cu", "score_kernels.cu",
            "accept_persistent.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler",
               "-fPIC", "--use_fast_math=false"]

@@ -198,10 +198,13 @@ int forward(hbsjd_ctx* c, int S, bool want_logits, int stop_layer = -1, int stop
         {
             const int ps = prof_begin(c, HBSJD_PROF_ATTENTION, 0.0);
             if constexpr (std::is_same<TA, bf16>::value) {
-                if (!c->ref_attention && attention_mma_supported(st, kv))
-                    launch_attention_mma(st, S, l, (const bf16*)c->q, kv, (bf16*)c->o, s);
-                else
+                if (!c->ref_attention && attention_tma_supported(st, kv)) {
+                    rc = launch_attention_tma(st, S, l, (const bf16*)c->q, Mcap, kv, (bf16*)c->o,
+                                              c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
+                    if (rc) return HBSJD_ECUDA;
+                } else {
                     launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
+                }
             } else {
                 launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
             }
@@ -338,7 +341,7 @@ int run_round(hbsjd_ctx* c) {
 
 void free_all(hbsjd_ctx* c) {
     void* ptrs[] = {c->w_img, c->rope_cs, c->kc, c->vc, c->page_table, c->st.cursor, c->st.seq, c->st.delta,
-                    c->st.qbase, c->st.label, c->st.klen, c->st.pfill, c->st.slot_img, c->st.slot_c, c->st.slot_n,
+                    c->st.qbase, c->st.label, c->st.klen, c->st.pfill, c->st.slot_img, c->st.slot_c, c->st.slot_n, c->st.slot_order,
                     c->st.counters, c->st.m_last, c->st.j_last, c->pbuf[0], c->pbuf[1], c->flag, c->cand_rep,
                     c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act,
                     c->stage_tok, c->stage_len, c->stage_lab, c->stage_out, c->verify_scratch,
@@ -465,6 +468,7 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
         (rc = dev_alloc(c, &st.label, Bm)) || (rc = dev_alloc(c, &st.klen, Bm)) ||
         (rc = dev_alloc(c, &st.pfill, Bm)) || (rc = dev_alloc(c, &st.slot_img, Bm)) ||
         (rc = dev_alloc(c, &st.slot_c, Bm)) || (rc = dev_alloc(c, &st.slot_n, Bm)) ||
+        (rc = dev_alloc(c, &st.slot_order, Bm)) ||
         (rc = dev_alloc(c, &st.counters, (size_t)8)) || (rc = dev_alloc(c, &st.m_last, Bm)) ||
         (rc = dev_alloc(c, &st.j_last, Bm)) || (rc = dev_alloc(c, &c->pbuf[0], Bm * Wm * V)) ||
         (rc = dev_alloc(c, &c->pbuf[1], Bm * Wm * V)) || (rc = dev_alloc(c, &c->flag, Bm * Wm)) ||

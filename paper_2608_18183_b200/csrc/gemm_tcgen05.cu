@@ -740,6 +740,10 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
 // 16 KB activation tile of every k-block has to cross from L2 whatever N is, and about 160 KB can be in flight
 // per SM); the epilogue adds about 0.15 us per 32 columns.  Large problems end up with 256 (CTA pairs), small
 // ones with the widest tile that still fits one wave.
+bool make_tensor_map_bf16(::CUtensorMap_st* map, const void* base, int rows, int cols, int box_rows) {
+    return make_map(map, base, rows, cols, box_rows);
+}
+
 int gemm_tcgen05_tile_n(int M, int N, int K) {
     const long tiles_m = (M + BM - 1) / BM;
     const int sms = 148, num_kb = K / BK;

@@ -6,6 +6,8 @@
 
 #include "common.cuh"
 
+struct CUtensorMap_st;  // CUtensorMap of <cuda.h>
+
 namespace hbsjd {
 
 // Device-side rollout state and per-round slot tables.  A "slot" is the place of one image in the
@@ -27,6 +29,7 @@ struct State {
     int32_t* slot_img; // [Bmax]
     int32_t* slot_c;   // [Bmax] first sequence index of the slot's inputs
     int32_t* slot_n;   // [Bmax] number of inputs (0: inactive slot)
+    int32_t* slot_order;  // [Bmax] slots by context length c + n, longest first (null: not built)
     int32_t* counters; // [8], see CNT_*
     int32_t* m_last;   // [Bmax] tokens committed in the last round
     int32_t* j_last;   // [Bmax] first-reject index of the last round (-1 none)
@@ -84,9 +87,11 @@ cudaError_t verify_enqueue(const VerifyDesc& d, const VerifyScratch& sc, const f
                            float* p_out, int32_t* cursor, int32_t* seq, uint8_t* delta, int32_t* qbase,
                            int32_t* m_out, cudaStream_t s);
 
-// ---- tensor-core ragged attention, bf16, head size 64 (attention_mma.cu)
-bool attention_mma_supported(const State& st, const KvView& kv);
-void launch_attention_mma(const State& st, int S, int layer, const bf16* q, KvView kv, bf16* out, cudaStream_t s);
+// ---- persistent tensor-core ragged attention, bf16, head size 64 (attention_tma.cu)
+bool attention_tma_supported(const State& st, const KvView& kv);
+// q_rows_cap: row capacity of the q buffer.  Returns 0 or a negative code with a message in err.
+int launch_attention_tma(const State& st, int S, int layer, const bf16* q, int q_rows_cap, KvView kv, bf16* out,
+                         int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
 
 // ---- state kernels (state_kernels.cu)
 void launch_init_state(const State& st, const int32_t* prefix_tokens, const int32_t* prefix_len,
@@ -130,6 +135,8 @@ void launch_score_reduce(int B, int T, const int32_t* prefix_len, const float* p
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
                      int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
 int gemm_tcgen05_tile_n(int M, int N, int K);
+// Cached TMA descriptor of a row-major bf16 matrix [rows, cols]: box = 64 columns x box_rows rows, 128-byte swizzle.
+bool make_tensor_map_bf16(::CUtensorMap_st* map, const void* base, int rows, int cols, int box_rows);
 // act[M, F] bf16 = silu(gate) * up, from A[M,K] . W13i^T where W13i[2F, K] holds gate row f at 2f, up row f at 2f+1.
 int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
                         int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);

@@ -65,6 +65,21 @@ __global__ void k_setup(State st, int phase, int compact) {
         if (tid == blockDim.x - 1) carry = before + incl;
         __syncthreads();
     }
+    // slots by context length, longest first (ties by slot index): the attention kernel deals its work items
+    // from this list so that every CTA streams about the same number of key blocks
+    if (st.slot_order != nullptr) {
+        __syncthreads();
+        const int n_slots = compact ? carry : st.B;
+        for (int s0 = tid; s0 < n_slots; s0 += blockDim.x) {
+            const int len = st.slot_n[s0] > 0 ? st.slot_c[s0] + st.slot_n[s0] : -1;
+            int rank = 0;
+            for (int s1 = 0; s1 < n_slots; ++s1) {
+                const int l1 = st.slot_n[s1] > 0 ? st.slot_c[s1] + st.slot_n[s1] : -1;
+                rank += (l1 > len) || (l1 == len && s1 < s0);
+            }
+            st.slot_order[rank] = s0;
+        }
+    }
     if (tid == 0) {
         st.counters[CNT_LIVE_SETUP] = carry;
         st.counters[CNT_SLOTS] = compact ? carry : st.B;
