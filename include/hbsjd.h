@@ -191,10 +191,23 @@ int hbsjd_debug_forward(hbsjd_ctx *c, int layer, int stage);
 /* Decoder GEMM as used by the round (Sec. 4.2 verifier forward): C[M,N] (+)= A[M,K] . W[N,K]^T on the
  * context's stream.  A, W: DEVICE, element type of the context (bf16: tcgen05 tensor cores, fp32
  * accumulation; fp32: CUDA cores).  C: DEVICE fp32 [M,N]; accumulate != 0 adds into C.
- * M may be any size; bf16 needs N % 64 == 0 and K % 64 == 0; A, W 16-byte aligned.  W is treated as a constant:
- * the kernel starts fetching it before earlier work of the stream has finished, so it must not be the output of a
- * library call still in flight on that stream (outputs of other kernels on the stream are ordered as usual). */
+ * M may be any size; bf16 needs N % 64 == 0 and K % 64 == 0; A, W 16-byte aligned.  A, W and C are ordered
+ * like any other kernel argument behind earlier work of the stream. */
 int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate);
+
+/* hbsjd_gemm `reps` times back to back before the one synchronisation (micro-benchmarks time the decoder's GEMM
+ * shapes the way a forward issues them), and -- acc_wait_ns > 0, bf16 contexts -- with the bounded wait of the
+ * epilogue warps on their accumulator shortened to that many nanoseconds (Sec. 4.2 verifier forward; the paper has
+ * no counterpart of the failure path).  A limit shorter than the main loop makes a healthy pipeline take the
+ * time-out path: every role leaves its loop, copies and MMAs in flight are drained, TMEM is freed, the call
+ * returns HBSJD_ETIMEOUT with C partly written, and the context stays usable.  Tests use it to exercise that path. */
+int hbsjd_debug_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate,
+                     int reps, unsigned int acc_wait_ns);
+
+/* Scatters the context's KV pages over the page pool (a seeded permutation of the page table) so that tests can
+ * check that results do not depend on where a row's pages lie (Sec. 4.2: per-image KV-cache locations).  Only
+ * before the first rollout of the context; HBSJD_ESTATE afterwards. */
+int hbsjd_debug_shuffle_pages(hbsjd_ctx *c, uint64_t seed);
 
 /* Probability pipeline of the verification step on caller-supplied logits (Sec. 4.2: "verification uses the
  * fused guided logits"): p = softmax(top_k((l_u + s (l_c - l_u)) / temperature)), ties at the k-th value kept.

@@ -163,7 +163,6 @@ def bench_probs(args):
 
 def bench_gemm(args):
     import torch
-    os.environ.setdefault("HBSJD_GEMM_NOSYNC", "1")  # hbsjd_gemm returns without waiting: launches run back to back
     from paper_2608_18183_b200 import binding, synth
     w = synth.WORKLOADS[args.workload]
     s = w.shape
@@ -178,8 +177,7 @@ def bench_gemm(args):
         Wt = (torch.randn(N, K, device="cuda", generator=g) * 0.05).bfloat16()
         Cm = torch.zeros(M, N, device="cuda")
         def burst():
-            for _ in range(20):
-                ctx.hbsjd_gemm(A, Wt, Cm, accumulate=bool(acc))
+            ctx.hbsjd_debug_gemm(A, Wt, Cm, accumulate=bool(acc), reps=20)  # 20 launches back to back, one sync
         us = _median_us(torch, burst, reps=5, warm=2) / 20
         print(json.dumps({"case": "gemm", "name": name, "M": M, "N": N, "K": K, "accumulate": acc,
                           "us": round(us, 1), "TFLOP_s": round(2.0 * M * N * K / us / 1e6, 1)}))

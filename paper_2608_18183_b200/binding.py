@@ -18,7 +18,8 @@ DBG_PROBS, DBG_LOGITS, DBG_SLOTS = 0, 1, 2
 DBG_ACT_A, DBG_ACT_Q, DBG_ACT_O, DBG_ACT_FFN, DBG_ACT_H, DBG_KV_K, DBG_KV_V = 3, 4, 5, 6, 7, 8, 9
 
 EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_profile_launch_floor", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
-           "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_debug_forward", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
+           "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_debug_forward", "hbsjd_debug_gemm",
+           "hbsjd_debug_shuffle_pages", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
            "hbsjd_last_error"]
 
 
@@ -101,6 +102,8 @@ def load():
         L.hbsjd_debug_read.argtypes = [vp, C.c_int, C.c_int, vp, C.c_size_t]
         L.hbsjd_debug_forward.argtypes = [vp, C.c_int, C.c_int]
         L.hbsjd_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int]
+        L.hbsjd_debug_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint]
+        L.hbsjd_debug_shuffle_pages.argtypes = [vp, C.c_uint64]
         L.hbsjd_bikl.argtypes = [vp, vp, vp, C.c_int, vp]
         L.hbsjd_score.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp, vp, C.POINTER(C.c_float)]
         L.hbsjd_strerror.argtypes = [C.c_int]
@@ -289,6 +292,18 @@ class Context:
         self._check(self.lib.hbsjd_gemm(self.h, A.data_ptr(), W.data_ptr(), Cout.data_ptr(), M, N, K,
                                         1 if accumulate else 0), "hbsjd_gemm")
         return Cout
+
+    def hbsjd_debug_gemm(self, A, W, Cout, accumulate=False, reps=1, acc_wait_ns=0):
+        """hbsjd_gemm `reps` times back to back; acc_wait_ns > 0 shortens the epilogue's bounded wait (time-out test)."""
+        M, K = A.shape
+        N = W.shape[0]
+        assert W.shape[1] == K and tuple(Cout.shape) == (M, N) and Cout.dtype == self._torch.float32
+        self._check(self.lib.hbsjd_debug_gemm(self.h, A.data_ptr(), W.data_ptr(), Cout.data_ptr(), M, N, K,
+                                              1 if accumulate else 0, reps, acc_wait_ns), "hbsjd_debug_gemm")
+        return Cout
+
+    def hbsjd_debug_shuffle_pages(self, seed: int):
+        self._check(self.lib.hbsjd_debug_shuffle_pages(self.h, seed), "hbsjd_debug_shuffle_pages")
 
     def hbsjd_bikl(self, logits_s, logits_t):
         """Device fp32 [rows, V] logits of two models -> device fp32 [rows] bidirectional KL (Eq. 3)."""

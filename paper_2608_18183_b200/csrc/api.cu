@@ -137,11 +137,14 @@ KvView kv_view(const hbsjd_ctx* c) {
 }
 
 // m_cap: row capacity of the A and C buffers when they are the context's own (0: exactly M rows)
+// w_constant: W is one of the model's weight matrices (see gemm_tcgen05_run)
 template <typename TA>
-int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int m_cap = 0);
+int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int m_cap = 0,
+         int w_constant = 1, unsigned int acc_wait_ns = 0);
 
 template <>
-int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int) {
+int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int, int,
+                unsigned int) {
     const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
     launch_gemm_simt<float>((const float*)A, (const float*)W, C, M, N, K, accumulate, c->stream);
     prof_end(c, ps);
@@ -151,11 +154,12 @@ int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int
 
 template <>
 int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
-               int m_cap) {
+               int m_cap, int w_constant, unsigned int acc_wait_ns) {
     c->launches++;
     const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
     const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, 0, m_cap,
-                                    c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err));
+                                    c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err), w_constant,
+                                    acc_wait_ns);
     prof_end(c, ps);
     return rc == 0 ? 0 : (rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA);
 }
@@ -445,15 +449,6 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
     {
         std::vector<int32_t> tab(c->n_pages);
         for (int i = 0; i < c->n_pages; ++i) tab[i] = i;
-        const char* sh = getenv("HBSJD_PAGE_SHUFFLE");
-        if (sh && atoi(sh) != 0) {  // scatter the pages (exercises the page-table indirection)
-            uint64_t x = 0x9E3779B97F4A7C15ull * (uint64_t)atoi(sh);
-            for (int i = c->n_pages - 1; i > 0; --i) {
-                x = x * 6364136223846793005ull + 1442695040888963407ull;
-                const int j = (int)((x >> 33) % (uint64_t)(i + 1));
-                std::swap(tab[i], tab[j]);
-            }
-        }
         CK(cudaMalloc((void**)&c->page_table, tab.size() * sizeof(int32_t)));
         CK(cudaMemcpyAsync(c->page_table, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice,
                            c->stream));
@@ -558,8 +553,7 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     c->Bmax = max_batch;
     c->Wmax = max_window;
     c->bf16_model = m->dtype == HBSJD_DTYPE_BF16;
-    const char* at = getenv("HBSJD_ATTENTION");
-    c->ref_attention = at && strcmp(at, "ref") == 0;
+    c->ref_attention = false;
     c->stream = (cudaStream_t)cuda_stream;
     c->dbg_layer = -1;
     c->err[0] = 0;
@@ -1118,13 +1112,39 @@ int hbsjd_debug_read(hbsjd_ctx* c, int what, int index, void* host_dst, size_t m
 }
 
 int hbsjd_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
-    if (!c || !A || !W || !C || M < 1 || N < 1 || K < 1) return HBSJD_EINVAL;
-    int rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate) : gemm<float>(c, A, W, C, M, N, K, accumulate);
-    if (rc) return rc;
+    return hbsjd_debug_gemm(c, A, W, C, M, N, K, accumulate, 1, 0);
+}
+
+int hbsjd_debug_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
+                     int reps, unsigned int acc_wait_ns) {
+    if (!c || !A || !W || !C || M < 1 || N < 1 || K < 1 || reps < 1) return HBSJD_EINVAL;
+    for (int r = 0; r < reps; ++r) {
+        // W is the caller's buffer, possibly written by earlier work of the stream: no early fetch of its tiles
+        const int rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate, 0, 0, acc_wait_ns)
+                                     : gemm<float>(c, A, W, C, M, N, K, accumulate);
+        if (rc) return rc;
+    }
     CK(cudaGetLastError());
-    static const bool nosync = getenv("HBSJD_GEMM_NOSYNC") != nullptr;  // tuning aid: back-to-back launches
-    if (nosync) return HBSJD_OK;
     return sync_counters(c);
+}
+
+int hbsjd_debug_shuffle_pages(hbsjd_ctx* c, uint64_t seed) {
+    if (!c) return HBSJD_EINVAL;
+    if (c->have_rollout) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_debug_shuffle_pages: only before the first rollout of the context");
+        return HBSJD_ESTATE;
+    }
+    std::vector<int32_t> tab(c->n_pages);
+    for (int i = 0; i < c->n_pages; ++i) tab[i] = i;
+    uint64_t x = 0x9E3779B97F4A7C15ull * (seed | 1ull);
+    for (int i = c->n_pages - 1; i > 0; --i) {
+        x = x * 6364136223846793005ull + 1442695040888963407ull;
+        const int j = (int)((x >> 33) % (uint64_t)(i + 1));
+        std::swap(tab[i], tab[j]);
+    }
+    CK(cudaMemcpyAsync(c->page_table, tab.data(), tab.size() * sizeof(int32_t), cudaMemcpyHostToDevice, c->stream));
+    CK(cudaStreamSynchronize(c->stream));
+    return HBSJD_OK;
 }
 
 }  // extern "C"

@@ -47,7 +47,8 @@ struct GemmArgs {
     bf16* out;       // SWIGLU: [M, N/2];  QKV: q [M, D]
     int M, N, K;
     int32_t* error_flag;
-    unsigned long long* timeline;  // tuning aid: when set, CTA 0 records %globaltimer stamps of its phases
+    int w_constant;   // W never changes while the stream runs (model weights): its tiles may be fetched early
+    unsigned int acc_wait_ns;  // 0, or a shorter limit for the epilogue's accumulator wait (time-out test)
     // QKV epilogue
     State st;
     int S, layer;
@@ -82,17 +83,21 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait (about one second).  Returns false when it gave up or another role raised `abort`.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort) {
+// Bounded wait (about one second unless a shorter limit is given).  Returns false when it gave up or another
+// role raised `abort`.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort,
+                                          unsigned long long limit_ns = 1000000000ull) {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
+    const int polls = limit_ns < 1000000ull ? 1 : 128;  // a short limit is checked after every poll
     for (;;) {
-        for (int it = 0; it < 128; ++it)
+        for (int it = 0; it < polls; ++it)
             if (mbar_try(bar, parity)) return true;
         if (*abort) return false;
-        if (globaltimer_ns() - t0 > 1000000000ull) return false;
+        if (globaltimer_ns() - t0 > limit_ns) return false;
     }
 }
+
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -119,6 +124,15 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank) {
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
+}
+// Raises the CTA's abort flag and, in a CTA pair, the partner's, so that neither spends its own time-outs.
+template <bool PAIR>
+__device__ __forceinline__ void raise_abort(volatile uint32_t* abort_flag, uint32_t rank) {
+    *abort_flag = 1;
+    if (PAIR) {
+        const uint32_t remote = map_to_rank(smem_u32((const void*)abort_flag), rank ^ 1u);
+        asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(remote), "r"(1u) : "memory");
+    }
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -205,6 +219,7 @@ struct Cfg {
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;  // two accumulators
     static constexpr int STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffers x (32 rows x 128 bytes)
     static constexpr int SMEM = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static_assert(16 * STAGES + 32 + 8 + 8 <= 256, "barrier area");
 };
 
 // Per-row context of the QKV epilogue: where the token row's q / k / v go.
@@ -222,8 +237,6 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     using cfg = Cfg<BN, PAIR>;
     extern __shared__ unsigned char smem_raw[];
     pdl_trigger();
-    unsigned long long* tl = (g.timeline && blockIdx.x == 0) ? g.timeline : nullptr;
-    if (tl && threadIdx.x == 0) tl[0] = globaltimer_ns();  // kernel entry
     const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader of the pair
     const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;  // tile walker id
     const int units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
@@ -238,6 +251,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     const uint32_t accf0 = bars + 16 * cfg::STAGES, acce0 = accf0 + 16;
     volatile uint32_t* tmem_slot = (volatile uint32_t*)(bars_ptr + 16 * cfg::STAGES + 32);
     volatile uint32_t* abort_flag = tmem_slot + 1;
+    const uint32_t drain_bar = acce0 + 16 + 8;  // behind the tmem slot and the abort flag: used on the abort path only
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int M = g.M, N = g.N;
@@ -254,6 +268,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
             mbar_init(accf0 + 8 * b, 1);
             mbar_init(acce0 + 8 * b, PAIR ? 8 : 4);  // one arrival per epilogue warp (of both CTAs)
         }
+        mbar_init(drain_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -282,14 +297,13 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     if (PAIR) cluster_sync_all();  // both CTAs' barriers are initialised before either signals the other
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_base = *tmem_slot;
-    if (tl && threadIdx.x == 0) tl[1] = globaltimer_ns();  // set-up done
     // Everything above is on-chip set-up.  The weight operand W is constant for the life of the model, so the
     // producer thread fetches the W tiles of its first stages BEFORE the grid dependency resolves (they cross
     // HBM while the previous kernel drains); activations, outputs and slot tables are touched only after it.
     const bool is_producer = warp == 0 && lane == 0;
     const int num_groups = (num_kb + cfg::KG - 1) / cfg::KG;  // barrier groups per tile
     int prefetched = 0;  // groups of the first tile whose W tiles are already in flight
-    if (is_producer) {
+    if (is_producer && g.w_constant) {
         const int tile = unit;  // every CTA owns at least one tile
         const int n0 = (tile % tiles_n) * BN + (PAIR ? (int)rank * (BN / 2) : 0);
         prefetched = num_groups < cfg::GROUPS ? num_groups : cfg::GROUPS;
@@ -305,7 +319,6 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         }
     }
     pdl_wait();
-    if (tl && threadIdx.x == 0) tl[2] = globaltimer_ns();  // grid dependency released
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
@@ -324,7 +337,7 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     // are on the way; only the activation tiles are missing
                     if (!first_rev) {
                         if (!mbar_wait(empty0 + 8 * gs, ph ^ 1u, abort_flag)) {
-                            *abort_flag = 1;
+                            raise_abort<PAIR>(abort_flag, rank);
                             atomicExch(g.error_flag, 1);
                             ok = false;
                             break;
@@ -345,6 +358,20 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 }
                 if (!ok) break;
             }
+            if (*abort_flag) {
+                // Leaving early: the copies this thread issued must have landed before the CTA gives up its shared
+                // memory.  The groups armed last are the only ones that can still be in flight; their barriers
+                // complete when the bytes arrive whether or not anyone consumes them (in a pair they live in the
+                // leader, which waits for both CTAs' bytes; the end-of-kernel cluster barrier holds the partner).
+                if (!PAIR || rank == 0) {
+                    const uint32_t first = gc > (uint32_t)cfg::GROUPS ? gc - cfg::GROUPS : 0u;
+                    for (uint32_t g2 = first; g2 < gc; ++g2) {
+                        const unsigned long long t0 = globaltimer_ns();
+                        while (!mbar_try(full0 + 8 * (g2 % cfg::GROUPS), (g2 / cfg::GROUPS) & 1u))
+                            if (globaltimer_ns() - t0 > 1000000000ull) break;
+                    }
+                }
+            }
         }
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
@@ -364,7 +391,6 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                         ok = false;
                         break;
                     }
-                    if (tl && gc == 0) tl[3] = globaltimer_ns();  // first operands landed
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     // descriptors by increments of the 14-bit start-address field (16-byte units; the ring lies
                     // below 256 KB, so the field never carries): + STAGE_BYTES per k-block, + 32 bytes per MMA
@@ -385,13 +411,25 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     else umma_commit(empty0 + 8 * gs);
                 }
                 if (!ok) {
-                    *abort_flag = 1;
+                    raise_abort<PAIR>(abort_flag, rank);
                     atomicExch(g.error_flag, 2);
                     break;
                 }
                 if (PAIR) umma_commit_pair(accf0 + 8 * buf);  // accumulator complete
                 else umma_commit(accf0 + 8 * buf);
-                if (tl && j == 0) tl[4] = globaltimer_ns();  // first tile's MMAs issued
+            }
+            if (*abort_flag) {
+                // Leaving early: the MMAs issued so far must have completed before TMEM and the operand ring are
+                // released.  A commit on a barrier of its own completes when they have.
+                if (PAIR)
+                    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(
+                                     drain_bar)
+                                 : "memory");
+                else
+                    umma_commit(drain_bar);
+                const unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try(drain_bar, 0u))
+                    if (globaltimer_ns() - t0 > 1000000000ull) break;
             }
         }
     } else {
@@ -401,15 +439,14 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         for (int tile = unit; tile < num_tiles; tile += units, ++j) {
             const int m0 = (tile / tiles_n) * TM + (int)rank * BM, n0 = (tile % tiles_n) * BN;
             const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
-            if (!mbar_wait(accf0 + 8 * buf, aph, abort_flag)) {
+            if (!mbar_wait(accf0 + 8 * buf, aph, abort_flag, g.acc_wait_ns ? g.acc_wait_ns : 1000000000ull)) {
                 if (lane == 0) {
-                    *abort_flag = 1;
+                    raise_abort<PAIR>(abort_flag, rank);
                     atomicExch(g.error_flag, 3);
                 }
                 break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            if (tl && j == 0 && warp == 2 && lane == 0) tl[5] = globaltimer_ns();  // first accumulator ready
             const int row = m0 + quarter * 32 + lane;
             const uint32_t tbase = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
 
@@ -530,15 +567,12 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         }
         // the staging tiles must have been read before shared memory is released; the global writes
         // themselves complete like any other store before dependent kernels pass their grid dependency
-        if (tl && warp == 2 && lane == 0) tl[6] = globaltimer_ns();  // last epilogue chunk issued
         if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-        if (tl && warp == 2 && lane == 0) tl[7] = globaltimer_ns();  // staging drained
     }
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (PAIR) cluster_sync_all();  // neither CTA leaves while the other may still read its tiles or barriers
-    if (tl && threadIdx.x == 0) tl[8] = globaltimer_ns();  // all roles done
     if (warp == 1) {
         if (PAIR)
             asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
@@ -696,8 +730,10 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
                  M, N, K);
         return -1;
     }
-    static const int env_bn = getenv("HBSJD_GEMM_BN") ? atoi(getenv("HBSJD_GEMM_BN")) : 0;  // tuning aid
-    if (!force_bn && env_bn && N % env_bn == 0) force_bn = env_bn;
+    if (force_bn != 0 && force_bn != 32 && force_bn != 64 && force_bn != 128 && force_bn != 256) {
+        snprintf(err, errlen, "gemm: tile width %d is not one of 32, 64, 128, 256", force_bn);
+        return -1;
+    }
     int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N, K);
     while (bn > max_bn) bn >>= 1;
     if (bn < 32 || N % bn != 0) {
@@ -705,8 +741,7 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
         return -1;
     }
     // large problems: 256 x 256 tiles on CTA pairs (a third less operand traffic per FLOP)
-    static const bool pair_on = !(getenv("HBSJD_GEMM_PAIR") && atoi(getenv("HBSJD_GEMM_PAIR")) == 0);
-    const bool pair = pair_on && bn == 256 && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2;
+    const bool pair = !force_bn && bn == 256 && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2;
     CUtensorMap ma, mw, mc;
     memset(&mc, 0, sizeof(mc));
     const int map_rows = m_cap >= M ? m_cap : M;
@@ -746,7 +781,7 @@ bool make_tensor_map_bf16(::CUtensorMap_st* map, const void* base, int rows, int
 
 int gemm_tcgen05_tile_n(int M, int N, int K) {
     const long tiles_m = (M + BM - 1) / BM;
-    const int sms = 148, num_kb = K / BK;
+    const int sms = num_sms(), num_kb = K / BK;
     // enough 256-wide tiles for every SM: the wide tile has the lowest operand traffic per FLOP
     if (N % 256 == 0 && tiles_m * (N / 256) >= sms) return 256;
     int best = 0;
@@ -766,7 +801,8 @@ int gemm_tcgen05_tile_n(int M, int N, int K) {
 }
 
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
-                     int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+                     int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen, int w_constant,
+                     unsigned int acc_wait_ns) {
     if ((uintptr_t)C & 15) {
         snprintf(err, errlen, "gemm: C must be 16-byte aligned");
         return -1;
@@ -777,22 +813,8 @@ int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K
     g.N = N;
     g.K = K;
     g.error_flag = error_flag;
-    static unsigned long long* tl_dev = nullptr;
-    static const bool tl_on = getenv("HBSJD_GEMM_TIMELINE") != nullptr;
-    if (tl_on) {  // tuning aid: print the phase stamps of CTA 0 of this launch
-        if (!tl_dev) cudaMalloc((void**)&tl_dev, 16 * sizeof(unsigned long long));
-        cudaMemsetAsync(tl_dev, 0, 16 * sizeof(unsigned long long), s);
-        g.timeline = tl_dev;
-        const int rc = run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, m_cap, s, err, errlen);
-        unsigned long long h[16];
-        cudaMemcpyAsync(h, tl_dev, sizeof(h), cudaMemcpyDeviceToHost, s);
-        cudaStreamSynchronize(s);
-        fprintf(stderr, "gemm M%d N%d K%d acc%d timeline(ns): setup %llu wait %llu first_load %llu mma_issued %llu "
-                        "acc_ready %llu epi_issued %llu drained %llu done %llu\n",
-                M, N, K, accumulate, h[1] - h[0], h[2] - h[0], h[3] - h[0], h[4] - h[0], h[5] - h[0], h[6] - h[0],
-                h[7] - h[0], h[8] - h[0]);
-        return rc;
-    }
+    g.w_constant = w_constant;
+    g.acc_wait_ns = acc_wait_ns;
     return run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, m_cap, s, err, errlen);
 }
 
@@ -804,6 +826,7 @@ int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, i
     g.N = F2;
     g.K = K;
     g.error_flag = error_flag;
+    g.w_constant = 1;
     return run(EPI_SWIGLU, A, W13_interleaved, g, 0, 256, m_cap, s, err, errlen);
 }
 
@@ -816,6 +839,7 @@ int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, 
     g.N = 3 * st.D;
     g.K = st.D;
     g.error_flag = error_flag;
+    g.w_constant = 1;
     g.st = st;
     g.S = S;
     g.layer = layer;

@@ -132,8 +132,11 @@ void launch_score_reduce(int B, int T, const int32_t* prefix_len, const float* p
 // error_flag: device int set non-zero if a bounded pipeline wait gave up.  Returns 0, or a negative
 // code with a message in err.
 // m_cap (>= M, or 0): row capacity of the A and C buffers; lets one cached tensor map serve every M.
+// w_constant: W is a model weight (never written while the stream runs), so its first tiles may be fetched before
+// the preceding kernel has finished.  acc_wait_ns: 0, or a shorter limit of the epilogue's accumulator wait.
 int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K, int accumulate, int force_bn,
-                     int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
+                     int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen, int w_constant = 1,
+                     unsigned int acc_wait_ns = 0);
 int gemm_tcgen05_tile_n(int M, int N, int K);
 // Cached TMA descriptor of a row-major bf16 matrix [rows, cols]: box = 64 columns x box_rows rows, 128-byte swizzle.
 bool make_tensor_map_bf16(::CUtensorMap_st* map, const void* base, int rows, int cols, int box_rows);

@@ -72,3 +72,29 @@ def test_fp32_gemm(ctx_fp32, M, N, K):
     ctx_fp32.hbsjd_gemm(A, W, C)
     ref = (A.double() @ W.double().T).float()
     assert float((C - ref).abs().max()) < 1e-5 * K ** 0.5
+
+
+def test_bounded_wait_runs_out_and_the_context_recovers(ctx_bf16):
+    """The failure path of the GEMM pipeline on a healthy GPU: the epilogue warps' bounded wait for their
+    accumulator is shortened to 300 ns while the main loop over K = 8192 needs tens of microseconds, so the wait
+    runs out.  The kernel must not hang or fault: it raises its error flag, every role leaves its loop, the copies
+    and MMAs in flight are drained, TMEM is freed, and the call returns HBSJD_ETIMEOUT (-5).  The next call on the
+    same context runs normally and is correct.  (One CTA per tile: the shape is too small for CTA pairs.)"""
+    import torch
+    g = torch.Generator(device="cuda").manual_seed(11)
+    M, N, K = 256, 256, 8192
+    A = (torch.randn(M, K, generator=g, device="cuda") * 0.5).bfloat16()
+    W = (torch.randn(N, K, generator=g, device="cuda") * 0.05).bfloat16()
+    C = torch.zeros(M, N, device="cuda")
+    with pytest.raises(binding.HbsjdError) as e:
+        ctx_bf16.hbsjd_debug_gemm(A, W, C, acc_wait_ns=300)
+    assert e.value.code == -5
+    torch.cuda.synchronize()
+    C2 = torch.zeros(M, N, device="cuda")
+    ctx_bf16.hbsjd_gemm(A, W, C2)
+    ref = A.float() @ W.float().T
+    assert float((C2 - ref).abs().max()) <= 2e-5 * max(float(ref.abs().max()), 1.0) * (K / 64) ** 0.5 + 1e-6
+    # several launches back to back through the same entry point give the same result as one
+    C3 = torch.zeros(M, N, device="cuda")
+    ctx_bf16.hbsjd_debug_gemm(A, W, C3, reps=3)
+    assert torch.equal(C3, C2)

@@ -133,7 +133,6 @@ def test_small_bf16_wide_windows_multi_page(W):
 def test_stepwise_equals_monolithic_and_modes_agree():
     """rollout(max_rounds=0) + rounds == one rollout call; Full == Compact == Hybrid bit for bit;
     scattered KV pages change nothing."""
-    import os
     w = synth.WORKLOADS["tiny_bf16"]
     toks, k, lab = synth.make_inputs(w)
     k[2] = w.shape.T  # finished from the start
@@ -161,11 +160,8 @@ def test_stepwise_equals_monolithic_and_modes_agree():
     assert n == st_full["rounds"]
     ctx.hbsjd_destroy()
     # scattered pages
-    os.environ["HBSJD_PAGE_SHUFFLE"] = "7"
-    try:
-        ctx2 = _ctx(w)
-    finally:
-        del os.environ["HBSJD_PAGE_SHUFFLE"]
+    ctx2 = _ctx(w)
+    ctx2.hbsjd_debug_shuffle_pages(7)
     out, _ = ctx2.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 3, exec_mode=binding.EXEC_HYBRID, gamma=3))
     np.testing.assert_array_equal(out.cpu().numpy(), ref)
     ctx2.hbsjd_destroy()
