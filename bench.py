@@ -33,6 +33,8 @@ UNIT = "tokens/s"
 # dram__bytes_write.sum, summarised under profiles/): mean over the 97 GEMM launches of one Full round of workload L.
 NCU_GEMM_TRAFFIC_BYTES_PER_LAUNCH = {"L": 54.9e6}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# nominal figures of the part, for context beside the measured denominators: dense bf16 tensor peak, HBM3e bandwidth
+NOMINAL_PEAKS = {"bf16_tflops": 2250.0, "hbm_gbs": 7700.0}
 
 
 def peaks():
@@ -98,8 +100,8 @@ def sample_plan(w, k):
     """Bounded oracle sample per workload: (image ids, rounds, description), sized for roughly 5-30 s of CPU
     work per step.  The large models take the images with the shortest prefixes (cheapest pre-filling)."""
     order = [int(i) for i in np.argsort(k, kind="stable")]
-    n_img, n_rounds = {"tiny": (w.batch, 0), "tiny_bf16": (w.batch, 0), "small_bf16": (w.batch, 0), "B": (4, 3),
-                       "L": (1, 2), "XL": (1, 1), "stress": (1, 2)}.get(w.name, (1, 1))
+    n_img, n_rounds = {"tiny": (w.batch, 0), "tiny_bf16": (w.batch, 0), "small_bf16": (w.batch, 0), "B": (8, 6),
+                       "L": (2, 4), "XL": (1, 3), "stress": (2, 4)}.get(w.name, (1, 1))
     ids = list(range(n_img)) if n_img == w.batch else order[:n_img]
     what = (f"{n_img} image(s) of the batch with the shortest prefixes (ids {ids}, prefix lengths "
             f"{[int(k[i]) for i in ids]}): prefix pre-filling + {n_rounds or 'all'} rounds")
@@ -290,7 +292,10 @@ def main():
             "avg_launch_ms": g["ms"] / max(g["launches"], 1), "launches": g["launches"],
             "share_of_step": g["ms"] / ms_prof if ms_prof > 0 else None,
             "event_pair_launch_floor_us": floor_us,
-            "frac_net_of_launch_floor": net(g) / 1e12 / pk["bf16_tflops_sustained"]}
+            "frac_net_of_launch_floor": net(g) / 1e12 / pk["bf16_tflops_sustained"],
+            "frac_of_measured_burst": gemm_tflops / pk["bf16_tflops"],
+            "frac_of_nominal": gemm_tflops / NOMINAL_PEAKS["bf16_tflops"],
+            "nominal_peak": NOMINAL_PEAKS["bf16_tflops"]}
     if w.shape.dtype != "bf16":
         roof.update(bound="alu", peak=72.0, peak_source="fp32 CUDA-core FMA: 148 SMs x 128 lanes x 2 x 1.9 GHz")
         roof["frac"] = gemm_tflops / 72.0
@@ -302,7 +307,8 @@ def main():
         other[name] = {"bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                        "frac": gbs / pk["hbm_gbs"], "ms_per_step": c["ms"] / args.steps,
                        "share_of_step": c["ms"] / ms_prof if ms_prof > 0 else None,
-                       "frac_net_of_launch_floor": net(c) / 1e9 / pk["hbm_gbs"]}
+                       "frac_net_of_launch_floor": net(c) / 1e9 / pk["hbm_gbs"],
+                       "frac_of_nominal": gbs / NOMINAL_PEAKS["hbm_gbs"], "nominal_peak": NOMINAL_PEAKS["hbm_gbs"]}
 
     value, total_tokens = job_tokens_per_s(tokens_per_step, args.steps, dist, "cuda", ms)
     committed = sum(s["committed"] for s in stats)
