@@ -170,7 +170,8 @@ int hbsjd_set_state(hbsjd_ctx *c, const int32_t *cursor, const int32_t *seq, con
  *   HBSJD_DBG_LOGITS  index = 2*image + branch (0 conditional, 1 unconditional): fp32 [window, V]
  *   HBSJD_DBG_SLOTS   index ignored: int32 [3, n_slots] = image, cursor, n of each physical slot; returns n_slots
  *   After hbsjd_debug_forward (index = 2*image + branch; elements of the context's type unless stated):
- *   HBSJD_DBG_ACT_A   [n, dim]  normed operand of the last projection that ran (QKV at stage 0, gate/up at stage 1)
+ *   HBSJD_DBG_ACT_A   [n, dim]  operand of the next projection: fp32 models, the normed rows of the last norm that ran;
+ *                     bf16 models (RMSNorm folded into the GEMMs), the bf16 copy of the residual stream
  *   HBSJD_DBG_ACT_Q   [n, dim]  rotated queries        HBSJD_DBG_ACT_O  [n, dim]  attention output
  *   HBSJD_DBG_ACT_FFN [n, ffn_hidden]  silu(gate) * up  HBSJD_DBG_ACT_H  fp32 [n, dim]  residual stream
  *   HBSJD_DBG_KV_K / HBSJD_DBG_KV_V  [cursor + n, dim]  cache rows of sequence indices 0..cursor+n-1 of that layer;
@@ -195,7 +196,10 @@ int hbsjd_debug_forward(hbsjd_ctx *c, int layer, int stage);
  * like any other kernel argument behind earlier work of the stream. */
 int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate);
 
-/* hbsjd_gemm `reps` times back to back before the one synchronisation (micro-benchmarks time the decoder's GEMM
+/* accumulate = 2 (bf16 contexts, N = dim, M within the context's activation rows): the residual-update form the
+ * forward itself uses, C += A W^T together with the bf16 copy and the per-row partial sums of squares of the new C
+ * (written to buffers of the context), so that it can be timed and checked alone.
+ * hbsjd_gemm `reps` times back to back before the one synchronisation (micro-benchmarks time the decoder's GEMM
  * shapes the way a forward issues them), and -- acc_wait_ns > 0, bf16 contexts -- with the bounded wait of the
  * epilogue warps on their accumulator shortened to that many nanoseconds (Sec. 4.2 verifier forward; the paper has
  * no counterpart of the failure path).  A limit shorter than the main loop makes a healthy pipeline take the
@@ -203,6 +207,16 @@ int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int 
  * returns HBSJD_ETIMEOUT with C partly written, and the context stays usable.  Tests use it to exercise that path. */
 int hbsjd_debug_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate,
                      int reps, unsigned int acc_wait_ns);
+
+/* Chooses the form of RMSNorm of a bf16 context (Sec. 4.2 verifier forward; the paper does not go below the model):
+ * on = 1 folds it into the GEMM epilogues (bf16 copy of the unnormalised residual stream as the operand, gain in the
+ * weights, row factor in the next epilogue), on = 0 runs it as a kernel of its own in front of the projections.
+ * hbsjd_create picks the folded form for contexts of at most 2048 activation rows (2 x max_batch x max_window) and the
+ * separate one above; this call lets tests run either form at any size.  The two forms round the GEMM operand at
+ * different points (x r g against x), so their results differ at bf16-noise level; one context always uses one form,
+ * so Full and Compact execution stay bit-identical.  Only before the first rollout, and only for models whose norm
+ * gains are all 1 (nothing to re-fold): HBSJD_ESTATE otherwise. */
+int hbsjd_debug_fold_norm(hbsjd_ctx *c, int on);
 
 /* Scatters the context's KV pages over the page pool (a seeded permutation of the page table) so that tests can
  * check that results do not depend on where a row's pages lie (Sec. 4.2: per-image KV-cache locations).  Only

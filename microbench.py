@@ -168,16 +168,20 @@ def bench_gemm(args):
     s = w.shape
     D, F, V = s.dim, s.ffn_hidden, s.vocab
     M = args.rows or w.batch * (2 if w.cfg_scale != 1.0 else 1) * w.window
-    ctx = _small_context(binding, synth, 64, 2, 4)
+    # a context of the workload's width (one thin layer): the residual-update form writes into its buffers
+    sh = synth.ModelShape(1, D, s.n_heads, 64, 64, 4, 4, 3, "bf16")
+    ctx = binding.Context(sh, synth.make_weights(sh, 3, target_entropy=None), (M + 63) // 64, 32)
     g = torch.Generator(device="cuda")
     g.manual_seed(args.seed)
-    for name, N, K, acc in [("qkv", 3 * D, D, 0), ("attention out (+=)", D, D, 1), ("gate|up", 2 * F, D, 0),
-                            ("down (+=)", D, F, 1), ("head", V, D, 0)]:
+    for name, N, K, acc in [("qkv", 3 * D, D, 0), ("attention out (+=)", D, D, 1),
+                            ("attention out (+=, bf16 copy, sums of squares)", D, D, 2), ("gate|up", 2 * F, D, 0),
+                            ("down (+=)", D, F, 1), ("down (+=, bf16 copy, sums of squares)", D, F, 2),
+                            ("head", V, D, 0)]:
         A = torch.randn(M, K, device="cuda", generator=g).bfloat16()
         Wt = (torch.randn(N, K, device="cuda", generator=g) * 0.05).bfloat16()
         Cm = torch.zeros(M, N, device="cuda")
         def burst():
-            ctx.hbsjd_debug_gemm(A, Wt, Cm, accumulate=bool(acc), reps=20)  # 20 launches back to back, one sync
+            ctx.hbsjd_debug_gemm(A, Wt, Cm, accumulate=acc, reps=20)  # 20 launches back to back, one sync
         us = _median_us(torch, burst, reps=5, warm=2) / 20
         print(json.dumps({"case": "gemm", "name": name, "M": M, "N": N, "K": K, "accumulate": acc,
                           "us": round(us, 1), "TFLOP_s": round(2.0 * M * N * K / us / 1e6, 1)}))

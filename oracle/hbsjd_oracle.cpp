@@ -106,6 +106,8 @@ struct Model {
     int acc_f32 = 0;      // dot products and sums of squares accumulate in fp32 instead of double
     int attn_w_bf16 = 0;  // the unnormalised attention weights are rounded to bf16 before they multiply the values
                           // (the usual tensor-core formulation; the normaliser keeps the unrounded weights)
+    int norm_folded = 0;  // RMSNorm(x) W^T evaluated as r (bf16(x) diag(g) W^T), r = rsqrt(mean(x^2) + eps): the row
+                          // factor applied after the product instead of before it (the same function of x)
     std::vector<float> tok_emb, cls_emb, g_out, w_head;
     std::vector<Layer> layers;
 };
@@ -167,6 +169,30 @@ void rmsnorm(const Model& M, const float* x, const float* g, float* out) {
     }
 }
 
+inline float maybe_bf16(const Model& M, float v) { return M.act_bf16 ? bf16_round(v) : v; }
+
+// Y[n][N] = RMSNorm(x; g) W^T for n rows; a[n][D] receives the operand of the product.  The definition (norm, round
+// the operand, multiply) unless the diagnostic norm_folded is set.
+void normed_projection(const Model& M, const float* x, const float* g, int n, const float* W, int N, float* a,
+                       float* Y) {
+    const int D = M.d.D;
+    if (!M.norm_folded) {
+        for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], g, &a[(size_t)i * D]);
+        matmul(M, a, n, D, W, N, Y);
+        return;
+    }
+    std::vector<double> r(n);
+    for (int i = 0; i < n; ++i) {
+        double ss = 0.0;
+        for (int k = 0; k < D; ++k) ss += (double)x[(size_t)i * D + k] * x[(size_t)i * D + k];
+        r[i] = 1.0 / std::sqrt(ss / D + (double)M.d.eps);
+        for (int k = 0; k < D; ++k) a[(size_t)i * D + k] = maybe_bf16(M, x[(size_t)i * D + k]) * g[k];
+    }
+    matmul(M, a, n, D, W, N, Y);
+    for (int i = 0; i < n; ++i)
+        for (int o = 0; o < N; ++o) Y[(size_t)i * N + o] = (float)((double)Y[(size_t)i * N + o] * r[i]);
+}
+
 // 2D rotary embedding on one head vector at sequence index s.
 // Index 0 (class token) is not rotated.  Index s >= 1 is image token s-1 at
 // (row, col) = ((s-1) / gw, (s-1) % gw).  Adjacent pairs (2e, 2e+1): the first
@@ -186,8 +212,6 @@ void rope2d(const Model& M, float* v, int s) {
         v[2 * e + 1] = (float)(a * sn + b * cs);
     }
 }
-
-inline float maybe_bf16(const Model& M, float v) { return M.act_bf16 ? bf16_round(v) : v; }
 
 void embed(const Model& M, int label, const int32_t* seq, int s, float* x) {
     const int D = M.d.D;
@@ -218,8 +242,7 @@ inline void trace_copy(float* dst, const float* src, size_t count) {
 void stage_ffn_act(const Model& M, const Layer& Ly, const float* x, int n, float* m, float* act) {
     const int D = M.d.D, F = M.d.F;
     std::vector<float> gu((size_t)n * 2 * F);
-    for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], Ly.g_ffn.data(), &m[(size_t)i * D]);
-    matmul(M, m, n, D, Ly.w_13.data(), 2 * F, gu.data());
+    normed_projection(M, x, Ly.g_ffn.data(), n, Ly.w_13.data(), 2 * F, m, gu.data());
     for (int i = 0; i < n; ++i)
         for (int f = 0; f < F; ++f) {
             const double g = gu[(size_t)i * 2 * F + f], u = gu[(size_t)i * 2 * F + F + f];
@@ -250,8 +273,7 @@ void ffn_block(const Model& M, const Layer& Ly, std::vector<float>& x, int n, co
 void head(const Model& M, const std::vector<float>& x, int n, float* logits) {
     const int D = M.d.D;
     std::vector<float> hn((size_t)n * D);
-    for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], M.g_out.data(), &hn[(size_t)i * D]);
-    matmul(M, hn.data(), n, D, M.w_head.data(), M.d.V, logits);
+    normed_projection(M, x.data(), M.g_out.data(), n, M.w_head.data(), M.d.V, hn.data(), logits);
 }
 
 // Attention of one query vector q (head h) at sequence index s over keys 0..s
@@ -298,8 +320,7 @@ void attend(const Model& M, const float* q, const float* K, const float* V, int 
 //     c+i, all three rounded (bf16): q is the query operand, k and v are the cache contents.
 void stage_qkv(const Model& M, const Layer& Ly, const float* x, int n, int c, float* a, float* qkv) {
     const int D = M.d.D, dh = M.dh, Hh = M.d.Hh;
-    for (int i = 0; i < n; ++i) rmsnorm(M, &x[(size_t)i * D], Ly.g_attn.data(), &a[(size_t)i * D]);  // (bf16)
-    matmul(M, a, n, D, Ly.w_qkv.data(), 3 * D, qkv);
+    normed_projection(M, x, Ly.g_attn.data(), n, Ly.w_qkv.data(), 3 * D, a, qkv);  // a: (bf16)
     for (int i = 0; i < n; ++i) {
         float* q = &qkv[(size_t)i * 3 * D];
         float* k = q + D;
@@ -750,9 +771,10 @@ void orc_stage_ffn_down(void* m, int layer, const float* act, int n, float* x) {
 }
 
 // Diagnostics for the noise-floor calibration (both 0: the oracle proper).  Never a comparison target.
-void orc_model_set_diag(void* m, int acc_f32, int attn_w_bf16) {
+void orc_model_set_diag(void* m, int acc_f32, int attn_w_bf16, int norm_folded) {
     ((Model*)m)->acc_f32 = acc_f32;
     ((Model*)m)->attn_w_bf16 = attn_w_bf16;
+    ((Model*)m)->norm_folded = norm_folded;
 }
 
 void orc_probs(const float* lc, const float* lu, float s, float tau, int k, int V, float* p) {

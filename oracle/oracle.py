@@ -59,7 +59,7 @@ def lib():
         L.orc_forward_window.argtypes = [vp, f32p, f32p, C.c_int, i32p, C.c_int, C.c_int, f32p]
         L.orc_forward_window_trace.argtypes = [vp, f32p, f32p, C.c_int, i32p, C.c_int, C.c_int, f32p,
                                                C.POINTER(Trace)]
-        L.orc_model_set_diag.argtypes = [vp, C.c_int, C.c_int]
+        L.orc_model_set_diag.argtypes = [vp, C.c_int, C.c_int, C.c_int]
         L.orc_stage_qkv.argtypes = [vp, C.c_int, f32p, C.c_int, C.c_int, f32p, f32p]
         L.orc_stage_attend.argtypes = [vp, f32p, f32p, f32p, C.c_int, C.c_int, f32p]
         L.orc_stage_attn_out.argtypes = [vp, C.c_int, f32p, C.c_int, f32p]
@@ -282,11 +282,12 @@ class Model:
         lib().orc_stage_ffn_down(self.h, layer, _p(act, C.c_float), act.shape[0], _p(x, C.c_float))
         return x
 
-    def set_diag(self, acc_f32: bool = False, attn_w_bf16: bool = False):
+    def set_diag(self, acc_f32: bool = False, attn_w_bf16: bool = False, norm_folded: bool = False):
         """Diagnostics of the noise-floor calibration, never a comparison target: accumulate dot products in fp32
-        instead of double; round the unnormalised attention weights to bf16 before they multiply the values.
+        instead of double; round the unnormalised attention weights to bf16 before they multiply the values;
+        apply RMSNorm's row factor after the projection (operand bf16(x) instead of bf16(x r g)).
         set_diag() restores the oracle proper."""
-        lib().orc_model_set_diag(self.h, int(acc_f32), int(attn_w_bf16))
+        lib().orc_model_set_diag(self.h, int(acc_f32), int(attn_w_bf16), int(norm_folded))
 
     def ar_rollout(self, prefix_tokens, prefix_len, labels, params: Params, image_ids=None) -> np.ndarray:
         pt, pl, lb = _i32(prefix_tokens), _i32(prefix_len), _i32(labels)

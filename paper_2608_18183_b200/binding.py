@@ -19,7 +19,7 @@ DBG_ACT_A, DBG_ACT_Q, DBG_ACT_O, DBG_ACT_FFN, DBG_ACT_H, DBG_KV_K, DBG_KV_V = 3,
 
 EXPORTS = ["hbsjd_create", "hbsjd_rollout", "hbsjd_rollout_host", "hbsjd_profile", "hbsjd_profile_read", "hbsjd_profile_launch_floor", "hbsjd_probs", "hbsjd_verify", "hbsjd_verify_static", "hbsjd_calibrate_gamma", "hbsjd_round", "hbsjd_tokens", "hbsjd_destroy", "hbsjd_get_state",
            "hbsjd_set_state", "hbsjd_debug_read", "hbsjd_debug_forward", "hbsjd_debug_gemm",
-           "hbsjd_debug_shuffle_pages", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
+           "hbsjd_debug_shuffle_pages", "hbsjd_debug_fold_norm", "hbsjd_gemm", "hbsjd_bikl", "hbsjd_score", "hbsjd_strerror",
            "hbsjd_last_error"]
 
 
@@ -104,6 +104,7 @@ def load():
         L.hbsjd_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int]
         L.hbsjd_debug_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint]
         L.hbsjd_debug_shuffle_pages.argtypes = [vp, C.c_uint64]
+        L.hbsjd_debug_fold_norm.argtypes = [vp, C.c_int]
         L.hbsjd_bikl.argtypes = [vp, vp, vp, C.c_int, vp]
         L.hbsjd_score.argtypes = [vp, vp, C.c_int, vp, vp, vp, vp, vp, C.POINTER(C.c_float)]
         L.hbsjd_strerror.argtypes = [C.c_int]
@@ -155,6 +156,8 @@ class Context:
         if rc != 0:
             raise HbsjdError(rc, "hbsjd_create", self.lib.hbsjd_strerror(rc).decode())
         self.max_batch, self.max_window = max_batch, max_window
+        # the library's rule for the form of RMSNorm of a bf16 context (see hbsjd_debug_fold_norm)
+        self.fold_norm = shape.dtype == "bf16" and 2 * max_batch * max_window <= 2048
         self.batch = 0
         self.window = 0
 
@@ -299,8 +302,13 @@ class Context:
         N = W.shape[0]
         assert W.shape[1] == K and tuple(Cout.shape) == (M, N) and Cout.dtype == self._torch.float32
         self._check(self.lib.hbsjd_debug_gemm(self.h, A.data_ptr(), W.data_ptr(), Cout.data_ptr(), M, N, K,
-                                              1 if accumulate else 0, reps, acc_wait_ns), "hbsjd_debug_gemm")
+                                              int(accumulate), reps, acc_wait_ns), "hbsjd_debug_gemm")
         return Cout
+
+    def hbsjd_debug_fold_norm(self, on: bool):
+        """RMSNorm folded into the GEMM epilogues (True) or as its own kernel (False); before the first rollout."""
+        self._check(self.lib.hbsjd_debug_fold_norm(self.h, 1 if on else 0), "hbsjd_debug_fold_norm")
+        self.fold_norm = bool(on)
 
     def hbsjd_debug_shuffle_pages(self, seed: int):
         self._check(self.lib.hbsjd_debug_shuffle_pages(self.h, seed), "hbsjd_debug_shuffle_pages")

@@ -26,6 +26,8 @@ struct hbsjd_ctx {
     hbsjd_model_desc d;
     int T, dh, Bmax, Wmax;
     bool bf16_model;
+    bool fold_norm;      // bf16 model: RMSNorm folded into the GEMM epilogues (launch-bound contexts), else its own kernel
+    bool unit_gains;     // every norm gain of the model is exactly 1
     bool ref_attention;  // debugging: run the one-warp-per-row attention kernel
     cudaStream_t stream;
     // weights
@@ -45,7 +47,8 @@ struct hbsjd_ctx {
     int32_t *cand_rep, *cand_ref;
     // activations
     float *h, *qkv, *gu, *logits;
-    void *a, *q, *o, *act;
+    void *a, *q, *o, *act;  // a: normed operand (fp32 model) / bf16 copy of the residual stream (bf16 model)
+    float* ssq;             // [rows][dim / 32] partial sums of squares of the residual rows (bf16 model)
     // host side
     int32_t* h_counters;  // pinned [8]
     cudaEvent_t ev0, ev1, ev2;
@@ -168,78 +171,143 @@ int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int 
 // stop_layer >= 0 (debugging): return after the attention sub-block (stop_stage 0) or the whole block
 // (stop_stage 1) of that layer, leaving the activation buffers as that point found them.
 template <typename TA>
-int forward(hbsjd_ctx* c, int S, bool want_logits, int stop_layer = -1, int stop_stage = 0) {
+int forward(hbsjd_ctx* c, int S, bool want_logits, int stop_layer = -1, int stop_stage = 0);
+
+// fp32 model: every step its own kernel (the configuration exists for parity, not speed).
+template <>
+int forward<float>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int stop_stage) {
+    typedef float TA;
     const State& st = c->st;
     const int M = st.nb * S * st.W, D = st.D, F = st.F;
-    const int Mcap = 2 * c->Bmax * c->Wmax;  // row capacity of the activation buffers
     cudaStream_t s = c->stream;
     const KvView kv = kv_view(c);
-    launch_embed<TA>(st, S, (const TA*)c->tok_emb, (const TA*)c->cls_emb, c->h, s);
+    launch_embed<TA>(st, S, (const TA*)c->tok_emb, (const TA*)c->cls_emb, c->h, nullptr, nullptr, s);
     c->launches++;
-    // RMSNorm of the fp32 residual stream into the GEMM operand; algorithmic bytes: read fp32, write TA
     auto norm = [&](const float* x, const void* gain) {
         const int ps = prof_begin(c, HBSJD_PROF_OTHER, (double)M * D * (4.0 + sizeof(TA)));
         launch_rmsnorm<TA>(x, (const TA*)gain, (TA*)c->a, M, D, c->d.rms_eps, s);
         prof_end(c, ps);
+        c->launches++;
     };
     for (int l = 0; l < st.L; ++l) {
         const LayerW& w = c->layers[l];
         int rc;
         norm(c->h, w.g_attn);
-        if constexpr (std::is_same<TA, bf16>::value) {
-            // QKV projection with RoPE and the paged KV write in its epilogue
-            const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D);
-            rc = gemm_tcgen05_qkv((const bf16*)c->a, (const bf16*)w.w_qkv, (bf16*)c->q, st, S, l, c->rope_cs, kv,
-                                  Mcap, c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
-            prof_end(c, ps);
-            if (rc) return rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
-            c->launches += 2;
-        } else {
-            if ((rc = gemm<TA>(c, c->a, w.w_qkv, c->qkv, M, 3 * D, D, 0))) return rc;
-            launch_rope_kv<TA>(st, S, l, c->qkv, c->rope_cs, (TA*)c->q, kv, s);
-            c->launches += 2;
-        }
+        if ((rc = gemm<TA>(c, c->a, w.w_qkv, c->qkv, M, 3 * D, D, 0))) return rc;
+        launch_rope_kv<TA>(st, S, l, c->qkv, c->rope_cs, (TA*)c->q, kv, s);
+        c->launches++;
         {
             const int ps = prof_begin(c, HBSJD_PROF_ATTENTION, 0.0);
-            if constexpr (std::is_same<TA, bf16>::value) {
-                if (!c->ref_attention && attention_tma_supported(st, kv)) {
-                    rc = launch_attention_tma(st, S, l, (const bf16*)c->q, Mcap, kv, (bf16*)c->o,
-                                              c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
-                    if (rc) return HBSJD_ECUDA;
-                } else {
-                    launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
-                }
-            } else {
-                launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
-            }
+            launch_attention_ref<TA>(st, S, l, (const TA*)c->q, kv, (TA*)c->o, s);
             prof_end(c, ps);
             c->launches++;
         }
-        if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1, Mcap))) return rc;
+        if ((rc = gemm<TA>(c, c->o, w.w_o, c->h, M, D, D, 1))) return rc;
         if (l == stop_layer && stop_stage == 0) return 0;
         norm(c->h, w.g_ffn);
+        if ((rc = gemm<TA>(c, c->a, w.w_13, c->gu, M, 2 * F, D, 0))) return rc;
+        launch_swiglu<TA>(c->gu, (TA*)c->act, M, F, s);
         c->launches++;
-        if constexpr (std::is_same<TA, bf16>::value) {
-            // gate/up projection with SwiGLU in its epilogue (gate and up rows interleaved at load time)
-            const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D);
-            rc = gemm_tcgen05_swiglu((const bf16*)c->a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D, Mcap,
-                                     c->st.counters + CNT_ERROR, s, c->err, sizeof(c->err));
-            prof_end(c, ps);
-            if (rc) return rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
-            c->launches++;
-        } else {
-            if ((rc = gemm<TA>(c, c->a, w.w_13, c->gu, M, 2 * F, D, 0))) return rc;
-            launch_swiglu<TA>(c->gu, (TA*)c->act, M, F, s);
-            c->launches++;
-        }
-        if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1, Mcap))) return rc;
+        if ((rc = gemm<TA>(c, c->act, w.w_2, c->h, M, D, F, 1))) return rc;
         if (l == stop_layer) return 0;
     }
     if (want_logits) {
         norm(c->h, c->g_out);
-        c->launches++;
         int rc;
-        if ((rc = gemm<TA>(c, c->a, c->w_head, c->logits, M, st.V, D, 0, Mcap))) return rc;
+        if ((rc = gemm<TA>(c, c->a, c->w_head, c->logits, M, st.V, D, 0))) return rc;
+    }
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        snprintf(c->err, sizeof(c->err), "forward launch: %s", cudaGetErrorString(e));
+        return HBSJD_ECUDA;
+    }
+    return 0;
+}
+
+// bf16 model: four tensor-core GEMMs and one attention kernel per layer; RoPE + the paged KV write, SwiGLU and the
+// residual add ride in the GEMM epilogues.  RMSNorm comes in two forms, fixed per context at creation:
+//   folded (contexts of at most 2048 activation rows, which are bound by the number of launches): no kernel of its
+//     own -- the kernels that write the residual stream (embedding gather, attention-out and FFN-down projections)
+//     also leave its bf16 copy and per-row partial sums of squares, the norm's gain is folded into the following
+//     weight matrix at load, and the following GEMM's epilogue applies the row factor rsqrt(mean(x^2) + eps);
+//   separate (larger contexts): one warp-per-row kernel in front of the QKV, gate/up and head projections, and the
+//     residual update as a bulk tensor reduce-add from the epilogue.  At 8192 rows the folded residual update costs
+//     what the separate kernel costs (its reads of the old residual compete with the operand stream for L2
+//     bandwidth), so the form with the exact operand rounding of the definition is kept there.
+template <>
+int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int stop_stage) {
+    const State& st = c->st;
+    const int M = st.nb * S * st.W, D = st.D, F = st.F;
+    const int Mcap = 2 * c->Bmax * c->Wmax;  // row capacity of the activation buffers
+    cudaStream_t s = c->stream;
+    const KvView kv = kv_view(c);
+    const bool fold = c->fold_norm;
+    bf16* a = (bf16*)c->a;  // folded: bf16 copy of the residual stream; separate: the normed operand
+    const NormIn nin = {fold ? c->ssq : nullptr, c->d.rms_eps};
+    int32_t* eflag = c->st.counters + CNT_ERROR;
+    auto done = [&](int rc) { return rc == 0 ? 0 : (rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA); };
+    auto norm = [&](const void* gain) {  // separate form only
+        const int ps = prof_begin(c, HBSJD_PROF_OTHER, (double)M * D * (4.0 + 2.0));
+        launch_rmsnorm<bf16>(c->h, (const bf16*)gain, a, M, D, c->d.rms_eps, s);
+        prof_end(c, ps);
+        c->launches++;
+    };
+    // residual update h += A W^T
+    auto residual = [&](const void* A, const void* W, int K) {
+        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * D * K);
+        int rc;
+        if (fold)
+            rc = gemm_tcgen05_addnorm((const bf16*)A, (const bf16*)W, c->h, a, c->ssq, M, D, K, Mcap, eflag, s, c->err,
+                                      sizeof(c->err));
+        else
+            rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, c->h, M, D, K, 1, 0, Mcap, eflag, s, c->err,
+                                  sizeof(c->err));
+        prof_end(c, ps);
+        c->launches++;
+        return rc;
+    };
+    launch_embed<bf16>(st, S, (const bf16*)c->tok_emb, (const bf16*)c->cls_emb, c->h, fold ? a : nullptr,
+                       fold ? c->ssq : nullptr, s);
+    c->launches++;
+    for (int l = 0; l < st.L; ++l) {
+        const LayerW& w = c->layers[l];
+        int rc, ps;
+        if (!fold) norm(w.g_attn);
+        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D);
+        rc = gemm_tcgen05_qkv(a, (const bf16*)w.w_qkv, (bf16*)c->q, st, S, l, c->rope_cs, kv, Mcap, nin, eflag, s,
+                              c->err, sizeof(c->err));
+        prof_end(c, ps);
+        if (rc) return done(rc);
+        ps = prof_begin(c, HBSJD_PROF_ATTENTION, 0.0);
+        if (attention_tma_supported(st, kv)) {
+            rc = launch_attention_tma(st, S, l, (const bf16*)c->q, Mcap, kv, (bf16*)c->o, eflag, s, c->err,
+                                      sizeof(c->err));
+            if (rc) return HBSJD_ECUDA;
+        } else {
+            launch_attention_ref<bf16>(st, S, l, (const bf16*)c->q, kv, (bf16*)c->o, s);
+        }
+        prof_end(c, ps);
+        c->launches += 2;
+        if ((rc = residual(c->o, w.w_o, D))) return done(rc);
+        if (l == stop_layer && stop_stage == 0) return 0;
+        if (!fold) norm(w.g_ffn);
+        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D);
+        rc = gemm_tcgen05_swiglu(a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D, Mcap, nin, eflag, s, c->err,
+                                 sizeof(c->err));
+        prof_end(c, ps);
+        if (rc) return done(rc);
+        c->launches++;
+        if ((rc = residual(c->act, w.w_2, F))) return done(rc);
+        if (l == stop_layer) return 0;
+    }
+    if (want_logits) {
+        if (!fold) norm(c->g_out);
+        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * st.V * D);
+        const int rc = gemm_tcgen05_head(a, (const bf16*)c->w_head, c->logits, M, st.V, D, Mcap, nin, eflag, s,
+                                         c->err, sizeof(c->err));
+        prof_end(c, ps);
+        if (rc) return done(rc);
+        c->launches++;
     }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
@@ -347,7 +415,7 @@ void free_all(hbsjd_ctx* c) {
     void* ptrs[] = {c->w_img, c->rope_cs, c->kc, c->vc, c->page_table, c->st.cursor, c->st.seq, c->st.delta,
                     c->st.qbase, c->st.label, c->st.klen, c->st.pfill, c->st.slot_img, c->st.slot_c, c->st.slot_n, c->st.slot_order,
                     c->st.counters, c->st.m_last, c->st.j_last, c->pbuf[0], c->pbuf[1], c->flag, c->cand_rep,
-                    c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act,
+                    c->cand_ref, c->h, c->qkv, c->gu, c->logits, c->a, c->q, c->o, c->act, c->ssq,
                     c->stage_tok, c->stage_len, c->stage_lab, c->stage_out, c->verify_scratch,
                     c->score_pos, c->score_img, c->score_loss, c->m_sync};
     for (void* p : ptrs)
@@ -391,16 +459,53 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
     CK(cudaMalloc((void**)&c->w_img, off));
     CK(cudaMemcpyAsync(c->w_img, weights, off, cudaMemcpyHostToDevice, c->stream));
     if (c->bf16_model) {
-        // the SwiGLU epilogue wants gate row f and up row f next to each other: rows (2f, 2f+1)
-        std::vector<uint16_t> tmp(2 * F * D);
+        // RMSNorm is folded around the GEMMs: W' = W diag(gain), rounded to bf16 once (exact when the gain is 1).
+        // Returns false when every gain is 1 and nothing has to be rewritten.
+        auto bf2f = [](uint16_t b) {
+            uint32_t u = (uint32_t)b << 16;
+            float f;
+            memcpy(&f, &u, 4);
+            return f;
+        };
+        auto f2bf = [](float f) {
+            uint32_t u;
+            memcpy(&u, &f, 4);
+            if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)(u >> 16);  // NaN
+            return (uint16_t)((u + 0x7fffu + ((u >> 16) & 1u)) >> 16);
+        };
+        c->unit_gains = true;
+        auto fold = [&](const uint16_t* W, const uint16_t* gain, size_t rows, std::vector<uint16_t>& out) {
+            bool ones = true;
+            for (size_t d = 0; d < D; ++d) ones = ones && gain[d] == 0x3f80;
+            c->unit_gains = c->unit_gains && ones;
+            if (ones || !c->fold_norm) return false;
+            out.resize(rows * D);
+            for (size_t r = 0; r < rows; ++r)
+                for (size_t d = 0; d < D; ++d) out[r * D + d] = f2bf(bf2f(W[r * D + d]) * bf2f(gain[d]));
+            return true;
+        };
+        const unsigned char* img = (const unsigned char*)weights;
+        std::vector<uint16_t> tmp(2 * F * D), folded;
         for (size_t l = 0; l < L; ++l) {
-            const uint16_t* src = (const uint16_t*)((const unsigned char*)weights + lo[l * 6 + 4]);
+            if (fold((const uint16_t*)(img + lo[l * 6 + 1]), (const uint16_t*)(img + lo[l * 6 + 0]), 3 * D, folded)) {
+                CK(cudaMemcpyAsync(c->w_img + lo[l * 6 + 1], folded.data(), folded.size() * 2, cudaMemcpyHostToDevice,
+                                   c->stream));
+                CK(cudaStreamSynchronize(c->stream));
+            }
+            // the SwiGLU epilogue wants gate row f and up row f next to each other: rows (2f, 2f+1)
+            const bool f13 = fold((const uint16_t*)(img + lo[l * 6 + 4]), (const uint16_t*)(img + lo[l * 6 + 3]), 2 * F,
+                                  folded);
+            const uint16_t* src = f13 ? folded.data() : (const uint16_t*)(img + lo[l * 6 + 4]);
             for (size_t f = 0; f < F; ++f) {
                 memcpy(&tmp[(2 * f) * D], src + f * D, D * 2);
                 memcpy(&tmp[(2 * f + 1) * D], src + (F + f) * D, D * 2);
             }
             CK(cudaMemcpyAsync(c->w_img + lo[l * 6 + 4], tmp.data(), tmp.size() * 2, cudaMemcpyHostToDevice,
                                c->stream));
+            CK(cudaStreamSynchronize(c->stream));
+        }
+        if (fold((const uint16_t*)(img + o_head), (const uint16_t*)(img + o_gout), V, folded)) {
+            CK(cudaMemcpyAsync(c->w_img + o_head, folded.data(), folded.size() * 2, cudaMemcpyHostToDevice, c->stream));
             CK(cudaStreamSynchronize(c->stream));
         }
     }
@@ -478,6 +583,7 @@ int create_impl(hbsjd_ctx* c, const void* weights, size_t weight_bytes) {
         (rc = dev_alloc(c, &a, Mmax * D * es)) || (rc = dev_alloc(c, &q, Mmax * D * es)) ||
         (rc = dev_alloc(c, &o, Mmax * D * es)) || (rc = dev_alloc(c, &act, Mmax * F * es)))
         return rc;
+    if ((rc = dev_alloc(c, &c->ssq, c->bf16_model ? Mmax * (D / 32) : (size_t)0))) return rc;
     c->a = a;
     c->q = q;
     c->o = o;
@@ -553,6 +659,8 @@ int hbsjd_create(hbsjd_ctx** out, const hbsjd_model_desc* m, const void* weights
     c->Bmax = max_batch;
     c->Wmax = max_window;
     c->bf16_model = m->dtype == HBSJD_DTYPE_BF16;
+    c->fold_norm = c->bf16_model && 2L * max_batch * max_window <= 2048;
+    c->unit_gains = false;
     c->ref_attention = false;
     c->stream = (cudaStream_t)cuda_stream;
     c->dbg_layer = -1;
@@ -1118,14 +1226,40 @@ int hbsjd_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int 
 int hbsjd_debug_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
                      int reps, unsigned int acc_wait_ns) {
     if (!c || !A || !W || !C || M < 1 || N < 1 || K < 1 || reps < 1) return HBSJD_EINVAL;
+    if (accumulate == 2 && (!c->bf16_model || N != c->d.dim || M > 2 * c->Bmax * c->Wmax)) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_debug_gemm: the residual-update form needs a bf16 context, N = dim and "
+                                         "M within the context's activation rows");
+        return HBSJD_EINVAL;
+    }
     for (int r = 0; r < reps; ++r) {
-        // W is the caller's buffer, possibly written by earlier work of the stream: no early fetch of its tiles
-        const int rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate, 0, 0, acc_wait_ns)
-                                     : gemm<float>(c, A, W, C, M, N, K, accumulate);
+        int rc;
+        if (accumulate == 2) {
+            // the form the forward uses for its residual updates: C += A W^T, plus the bf16 copy and the partial
+            // sums of squares of the new rows (into the context's own buffers)
+            c->launches++;
+            rc = gemm_tcgen05_addnorm((const bf16*)A, (const bf16*)W, C, (bf16*)c->a, c->ssq, M, N, K, 0,
+                                      c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err));
+            if (rc) rc = rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
+        } else {
+            // W is the caller's buffer, possibly written by earlier work of the stream: no early fetch of its tiles
+            rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate, 0, 0, acc_wait_ns)
+                               : gemm<float>(c, A, W, C, M, N, K, accumulate);
+        }
         if (rc) return rc;
     }
     CK(cudaGetLastError());
     return sync_counters(c);
+}
+
+int hbsjd_debug_fold_norm(hbsjd_ctx* c, int on) {
+    if (!c) return HBSJD_EINVAL;
+    if (!c->bf16_model || c->have_rollout || !c->unit_gains) {
+        snprintf(c->err, sizeof(c->err), "hbsjd_debug_fold_norm: needs a bf16 context with unit norm gains, before its "
+                                         "first rollout");
+        return HBSJD_ESTATE;
+    }
+    c->fold_norm = on != 0;
+    return HBSJD_OK;
 }
 
 int hbsjd_debug_shuffle_pages(hbsjd_ctx* c, uint64_t seed) {

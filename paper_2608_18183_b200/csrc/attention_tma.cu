@@ -1,14 +1,15 @@
 // Ragged attention over paged per-image KV caches (Sec. 4.2 "Batched verification"), bf16, head size 64:
-// persistent, warp-specialised, K/V and Q tiles moved by TMA.
+// persistent, warp-specialised, K/V blocks moved by TMA.
 //
 // Work item = one physical row (branch, slot) x HPC heads.  The items of a forward are dealt to the CTAs from a
 // list sorted by context length (longest first, alternate stripes reversed), so every CTA streams about the
 // same number of key blocks.  Inside a CTA
-//   warp 0 (one lane)   producer: for every item, the Q tile of each head, then the item's K and V blocks of 32
-//                       keys, each one cp.async.bulk.tensor copy (128-byte swizzle) into a ring of STAGES
-//                       stages, completion on mbarriers.  The producer runs ahead across item boundaries: the
-//                       next item's first blocks are in flight while the current item's last ones are used.
-//   warps 1..QB*HPC     consumers: warp (head, q-block) owns 16 consecutive window inputs of one head; online
+//   warp 0 (one lane)   producer: for every item, its K and V blocks of 32 keys, each one cp.async.bulk.tensor copy
+//                       (128-byte swizzle) into a ring of STAGES stages, completion on mbarriers.  The producer
+//                       runs ahead across item boundaries: the next item's first blocks are in flight while the
+//                       current item's last ones are used.
+//   warps 1..QB*HPC     consumers: warp (head, q-block) owns 16 consecutive window inputs of one head (its query
+//                       fragments come straight from global memory, once per item); online
 //                       softmax in fp32, products on mma.sync m16n8k16 (the work is about W FLOP per byte of K, V:
 //                       far below the tensor ridge, the tensor cores only keep the math off the critical path).
 // Query i of the row sits at sequence index s = c + i and attends keys 0..s: the cached prefix 0..c-1 plus the
@@ -109,6 +110,7 @@ struct AttnArgs {
     State st;
     int S, layer, G;  // slots, layer, head groups (heads / HPC)
     KvView kv;
+    const bf16* q;
     bf16* out;
     int32_t* error_flag;
 };
@@ -133,22 +135,18 @@ __device__ __forceinline__ bool item_at(const AttnArgs& a, const int* s_tab, int
 }
 
 template <int QB>
-__global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __grid_constant__ CUtensorMap map_q,
-                                                                       const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __grid_constant__ CUtensorMap map_k,
                                                                        const __grid_constant__ CUtensorMap map_v,
                                                                        const AttnArgs a) {
     pdl_trigger();
     constexpr int NCW = QB * HPC;                 // consumer warps
-    constexpr int Q_TILE = QB * 16 * DH * 2;      // Q tile of one head: QB * 2 KB
-    constexpr int Q_BYTES = HPC * Q_TILE;
     extern __shared__ unsigned char smem_raw[];
     const State& st = a.st;
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;               // [STAGES][HPC][K tile | V tile]
-    const uint32_t qbuf = ring + STAGES * STAGE_BYTES;          // [2][HPC][Q tile]
-    const uint32_t bars = qbuf + 2 * Q_BYTES;                   // full[STAGES], empty[STAGES], qfull[2], qempty[2]
-    const uint32_t full0 = bars, empty0 = bars + 8 * STAGES, qfull0 = bars + 16 * STAGES, qempty0 = qfull0 + 16;
-    unsigned char* tail = smem_raw + (bars - raw) + 16 * STAGES + 32;
+    const uint32_t bars = ring + STAGES * STAGE_BYTES;          // full[STAGES], empty[STAGES]
+    const uint32_t full0 = bars, empty0 = bars + 8 * STAGES;
+    unsigned char* tail = smem_raw + (bars - raw) + 16 * STAGES;
     volatile uint32_t* abort_flag = (volatile uint32_t*)tail;
     int* s_tab = (int*)(tail + 16);  // [4][S]: order, n, c, image of every slot
 
@@ -158,13 +156,8 @@ __global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __g
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, NCW);
         }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(qfull0 + 8 * b, 1);
-            mbar_init(qempty0 + 8 * b, NCW);
-        }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_q) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
     }
@@ -185,24 +178,12 @@ __global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __g
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
         if (lane == 0) {
-            uint32_t gc = 0, qc = 0;  // K/V stages and Q buffers issued so far
+            uint32_t gc = 0;  // K/V stages issued so far
             bool ok = true;
             for (int stripe = 0; ok && stripe * grid < n_items; ++stripe) {
                 const int pos = position(stripe);
                 Item it;
                 if (pos >= n_items || !item_at(a, s_tab, pos, it)) continue;
-                {   // Q tiles of the item's heads (rows past the window belong to the next row: never written back)
-                    const uint32_t qb = qc & 1u, qph = (qc >> 1) & 1u;
-                    if (!mbar_wait(qempty0 + 8 * qb, qph ^ 1u, abort_flag)) {
-                        ok = false;
-                        break;
-                    }
-                    mbar_expect_tx(qfull0 + 8 * qb, Q_BYTES);
-                    for (int h = 0; h < HPC; ++h)
-                        tma_load_2d(qbuf + qb * Q_BYTES + h * Q_TILE, &map_q, (it.head0 + h) * DH, it.prow * st.W,
-                                    qfull0 + 8 * qb);
-                    ++qc;
-                }
                 const int nblocks = (it.c + it.n + KB - 1) / KB;
                 const int32_t* pages = a.kv.table + (size_t)it.crow * a.kv.pages_per_row;
                 const int layer_row0 = a.layer * a.kv.n_pages * a.kv.page;
@@ -242,7 +223,7 @@ __global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __g
         // ---------------------------------------------------------------- consumers
         const int cw = warp - 1;
         const int wh = cw / QB, wq = cw % QB;  // head within the item, q-block
-        uint32_t gc = 0, qc = 0;
+        uint32_t gc = 0;
         const float sl2 = 0.125f * 1.4426950408889634f;  // 1/sqrt(64) * log2(e)
         bool ok = true;
         for (int stripe = 0; ok && stripe * grid < n_items; ++stripe) {
@@ -251,24 +232,22 @@ __global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __g
             if (pos >= n_items || !item_at(a, s_tab, pos, it)) continue;
             const int c = it.c, n = it.n;
             const int nblocks = (c + n + KB - 1) / KB;
-            // ---- this warp's queries: 16 rows x 64 dims as A fragments, from the Q tile
+            // ---- this warp's queries: 16 rows x 64 dims as A fragments.  Rows at or past n hold whatever the buffer
+            // holds (finite values of older forwards): their results are never written back.
+            const int i0 = wq * 16 + (lane >> 2), i1 = i0 + 8;
             uint32_t qa[4][4];
             {
-                const uint32_t qb = qc & 1u, qph = (qc >> 1) & 1u;
-                if (!mbar_wait(qfull0 + 8 * qb, qph, abort_flag)) {
-                    ok = false;
-                    break;
-                }
-                const uint32_t qt = qbuf + qb * Q_BYTES + wh * Q_TILE;
-                const int qrow = wq * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+                const bf16* qrow0 = a.q + ((size_t)it.prow * st.W + min(i0, st.W - 1)) * st.D + (it.head0 + wh) * DH;
+                const bf16* qrow1 = a.q + ((size_t)it.prow * st.W + min(i1, st.W - 1)) * st.D + (it.head0 + wh) * DH;
 #pragma unroll
-                for (int kc = 0; kc < 4; ++kc)
-                    ldmatrix_x4(qt + tile_off(qrow, kc * 2 + (lane >> 4)), qa[kc][0], qa[kc][1], qa[kc][2], qa[kc][3]);
-                __syncwarp();
-                if (lane == 0) mbar_arrive(qempty0 + 8 * qb);
-                ++qc;
+                for (int kc = 0; kc < 4; ++kc) {
+                    const int d = kc * 16 + (lane & 3) * 2;
+                    qa[kc][0] = *reinterpret_cast<const uint32_t*>(qrow0 + d);
+                    qa[kc][1] = *reinterpret_cast<const uint32_t*>(qrow1 + d);
+                    qa[kc][2] = *reinterpret_cast<const uint32_t*>(qrow0 + d + 8);
+                    qa[kc][3] = *reinterpret_cast<const uint32_t*>(qrow1 + d + 8);
+                }
             }
-            const int i0 = wq * 16 + (lane >> 2), i1 = i0 + 8;
             const bool warp_active = wq * 16 < n;  // q-blocks wholly past the window only keep the ring moving
             const int s0 = c + i0, s1 = c + i1;    // sequence index of this thread's two query rows
             float o[8][4];
@@ -400,10 +379,9 @@ __global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __g
 }
 
 template <int QB>
-cudaError_t launch_qb(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnArgs& a,
-                      cudaStream_t s) {
+cudaError_t launch_qb(const CUtensorMap& mk, const CUtensorMap& mv, const AttnArgs& a, cudaStream_t s) {
     constexpr int threads = (QB * HPC + 1) * 32;
-    const int smem = 1024 + STAGES * STAGE_BYTES + 2 * HPC * QB * 16 * DH * 2 + 16 * STAGES + 32 + 16 + 16 * a.S;
+    const int smem = 1024 + STAGES * STAGE_BYTES + 16 * STAGES + 16 + 16 * a.S;
     static int configured[64] = {0};
     cudaError_t e = ensure_dynamic_smem(k_attention_tma<QB>, smem, configured);
     if (e != cudaSuccess) return e;
@@ -414,7 +392,7 @@ cudaError_t launch_qb(const CUtensorMap& mq, const CUtensorMap& mk, const CUtens
     const long items = (long)a.S * a.st.nb * a.G;
     long grid = (long)device_sm_count() * per_sm;
     if (grid > items) grid = items;
-    return launch_k(k_attention_tma<QB>, dim3((unsigned)grid), dim3(threads), (size_t)smem, s, mq, mk, mv, a);
+    return launch_k(k_attention_tma<QB>, dim3((unsigned)grid), dim3(threads), (size_t)smem, s, mk, mv, a);
 }
 
 }  // namespace
@@ -425,11 +403,11 @@ bool attention_tma_supported(const State& st, const KvView& kv) {
 
 int launch_attention_tma(const State& st, int S, int layer, const bf16* q, int q_rows_cap, KvView kv, bf16* out,
                          int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mk, mv;
     const int qb = (st.W + 15) / 16;
     const long kv_rows = (long)st.L * kv.n_pages * kv.page;
-    if (kv_rows > 0x7fffffffL || !make_tensor_map_bf16(&mq, q, q_rows_cap, st.D, 16 * qb) ||
-        !make_tensor_map_bf16(&mk, kv.k, (int)kv_rows, st.D, KB) ||
+    (void)q_rows_cap;
+    if (kv_rows > 0x7fffffffL || !make_tensor_map_bf16(&mk, kv.k, (int)kv_rows, st.D, KB) ||
         !make_tensor_map_bf16(&mv, kv.v, (int)kv_rows, st.D, KB)) {
         snprintf(err, errlen, "attention: cuTensorMapEncodeTiled failed");
         return -3;
@@ -441,13 +419,14 @@ int launch_attention_tma(const State& st, int S, int layer, const bf16* q, int q
     a.G = st.Hh / HPC;
     a.kv = kv;
     a.out = out;
+    a.q = q;
     a.error_flag = error_flag;
     cudaError_t e;
     switch (qb) {
-        case 1: e = launch_qb<1>(mq, mk, mv, a, s); break;
-        case 2: e = launch_qb<2>(mq, mk, mv, a, s); break;
-        case 3: e = launch_qb<3>(mq, mk, mv, a, s); break;
-        default: e = launch_qb<4>(mq, mk, mv, a, s); break;
+        case 1: e = launch_qb<1>(mk, mv, a, s); break;
+        case 2: e = launch_qb<2>(mk, mv, a, s); break;
+        case 3: e = launch_qb<3>(mk, mv, a, s); break;
+        default: e = launch_qb<4>(mk, mv, a, s); break;
     }
     if (e != cudaSuccess) {
         snprintf(err, errlen, "attention launch: %s", cudaGetErrorString(e));

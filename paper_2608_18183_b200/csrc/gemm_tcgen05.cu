@@ -10,7 +10,9 @@
 // share its tile: Full and Compact execution give identical bits.
 //
 // Epilogues:  STORE  C fp32 = acc           (LM head -> logits)
-//             ADD    C fp32 += acc          (attention-out and FFN-down projections into the residual stream)
+//             ADD    C fp32 += acc          (public hbsjd_gemm with accumulate)
+//             ADDNORM  C fp32 += acc, bf16 copy of the new C, per-row partial sums of squares   (attention-out and
+//                    FFN-down projections into the residual stream; feeds the RMSNorm folded into the next GEMM)
 //             SWIGLU out bf16[M, N/2] = silu(acc[2f]) * acc[2f+1]   (gate/up rows interleaved at load time)
 //             QKV    2D RoPE on q and k, bf16 q[M, D], k and v written to the row's KV pages
 //
@@ -40,13 +42,22 @@ constexpr int BM = 128;
 constexpr int BK = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int NUM_THREADS = 192;
 
-enum { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2, EPI_QKV = 3 };
+enum { EPI_STORE = 0, EPI_ADD = 1, EPI_SWIGLU = 2, EPI_QKV = 3, EPI_ADDNORM = 4 };
 
 struct GemmArgs {
     float* C;        // STORE / ADD
     bf16* out;       // SWIGLU: [M, N/2];  QKV: q [M, D]
     int M, N, K;
     int32_t* error_flag;
+    // RMSNorm folded around the GEMMs (bf16 model): the operand A is the bf16 copy of the UNNORMALISED residual
+    // stream and the norm's gain is folded into W, so that norm(x) W^T = r (x W'^T) with the row factor
+    // r = rsqrt(mean(x^2) + eps) applied here, in the epilogue, from partial sums of squares
+    const float* ssq_in;   // [M][ssq_n] partial sums of squares of A's rows (null: no row factor)
+    int ssq_n;             // partials per row = K / 32
+    float inv_dim, eps;
+    // ADDNORM: C (fp32 residual) += acc, plus what the next GEMM needs
+    bf16* hb;              // [M][N] bf16 copy of the updated residual
+    float* ssq_out;        // [M][N / 32] sums of squares of the updated residual per 32-column chunk
     int w_constant;   // W never changes while the stream runs (model weights): its tiles may be fetched early
     unsigned int acc_wait_ns;  // 0, or a shorter limit for the epilogue's accumulator wait (time-out test)
     // QKV epilogue
@@ -205,21 +216,28 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 
 // PAIR: two CTAs of a cluster compute one 256 x BN tile with cta_group::2 MMAs; each CTA stages its own 128 rows
 // of A and its own BN/2 rows of W, which cuts the operand bytes per FLOP by a third against a 128 x BN tile.
-template <int BN, bool PAIR = false>
+// WIDE: the epilogue stages a bf16 tile beside every fp32 tile (EPI_ADDNORM), 48 KB instead of 32 KB; the operand
+// ring gives up a stage or two for it.
+template <int BN, bool PAIR = false, bool WIDE = false>
 struct Cfg {
-    // as many stages as fit beside the 32 KB epilogue staging: small tiles are latency-bound (one TMA round
-    // trip per ring revolution), so a narrow tile gets a deep ring
-    static constexpr int STAGES = PAIR ? 6 : (BN >= 256 ? 4 : (BN == 128 ? 6 : 8));
-    // k-blocks that share one full / empty barrier pair (one wait and one commit per 2 x 4 MMAs)
-    static constexpr int KG = (!PAIR && BN <= 64) ? 4 : 2;
+    // as many stages as fit beside the epilogue staging: small tiles are latency-bound (one TMA round trip per ring
+    // revolution), so a narrow tile gets a deep ring
+    static constexpr int STAGES = WIDE ? (PAIR ? 5 : (BN >= 256 ? 3 : (BN == 128 ? 5 : (BN == 64 ? 6 : 8))))
+                                       : (PAIR ? 6 : (BN >= 256 ? 4 : (BN == 128 ? 6 : 8)));
+    // k-blocks that share one full / empty barrier pair (one wait and one commit per KG x 4 MMAs)
+    static constexpr int KG = WIDE ? ((PAIR || BN >= 128) ? 1 : (BN == 64 ? 2 : 4)) : ((!PAIR && BN <= 64) ? 4 : 2);
     static constexpr int GROUPS = STAGES / KG;
+    static_assert(GROUPS * KG == STAGES && GROUPS >= 2, "ring stages must split into whole barrier groups");
     static constexpr int A_BYTES = BM * BK * 2;
     static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;  // two accumulators
-    static constexpr int STAGING_BYTES = 4 * 2 * 4096;  // 4 epilogue warps x 2 buffers x (32 rows x 128 bytes)
+    // 4 epilogue warps x 2 buffers x (32 rows x 128 bytes fp32 [+ 32 rows x 64 bytes bf16])
+    static constexpr int WARP_STAGING = WIDE ? 2 * 6144 : 2 * 4096;
+    static constexpr int STAGING_BYTES = 4 * WARP_STAGING;
     static constexpr int SMEM = STAGES * STAGE_BYTES + STAGING_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
     static_assert(16 * STAGES + 32 + 8 + 8 <= 256, "barrier area");
+    static_assert(SMEM <= 227 * 1024, "shared memory of one CTA");
 };
 
 // Per-row context of the QKV epilogue: where the token row's q / k / v go.
@@ -233,8 +251,9 @@ template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_constant__ CUtensorMap map_a,
                                                               const __grid_constant__ CUtensorMap map_w,
                                                               const __grid_constant__ CUtensorMap map_c,
+                                                              const __grid_constant__ CUtensorMap map_hb,
                                                               const GemmArgs g) {
-    using cfg = Cfg<BN, PAIR>;
+    using cfg = Cfg<BN, PAIR, EPI == EPI_ADDNORM>;
     extern __shared__ unsigned char smem_raw[];
     pdl_trigger();
     const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader of the pair
@@ -275,7 +294,9 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
     if (warp == 0 && lane == 0) {  // descriptor fetch off the critical path
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_a) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w) : "memory");
-        if (EPI == EPI_STORE || EPI == EPI_ADD) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+        if (EPI == EPI_STORE || EPI == EPI_ADD || EPI == EPI_ADDNORM)
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&map_c) : "memory");
+        if (EPI == EPI_ADDNORM) asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hb) : "memory");
     }
     if (warp == 1) {
         if (PAIR) {  // the same warp of both CTAs allocates the same columns in both
@@ -439,6 +460,41 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
         for (int tile = unit; tile < num_tiles; tile += units, ++j) {
             const int m0 = (tile / tiles_n) * TM + (int)rank * BM, n0 = (tile % tiles_n) * BN;
             const uint32_t buf = j & 1u, aph = (j >> 1) & 1u;
+            const int row = m0 + quarter * 32 + lane;
+            const uint32_t tbase = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
+            // what the tile's rows need from global memory is requested before the accumulator is waited for
+            // row factor of the folded RMSNorm: the partial sums of squares of this row of A, added in a fixed order
+            float rscale = 1.0f;
+            if (EPI != EPI_ADD && EPI != EPI_ADDNORM && g.ssq_in != nullptr && row < M) {
+                const float2* pp = reinterpret_cast<const float2*>(g.ssq_in + (size_t)row * g.ssq_n);
+                float ss = 0.f;
+                for (int v = 0; v < g.ssq_n / 2; ++v) {
+                    const float2 t = pp[v];
+                    ss += t.x;
+                    ss += t.y;
+                }
+                rscale = 1.0f / sqrtf(ss * g.inv_dim + g.eps);
+            }
+            // ADDNORM: the residual values this thread's row adds to, fetched three 32-column chunks ahead through a
+            // ring of four register buffers (a chunk is 128 contiguous bytes of the row; the first three are
+            // requested before the accumulator is waited for)
+            constexpr int UNR = EPI == EPI_ADDNORM ? 4 : 1;  // chunks per unrolled group: static ring indices
+            float4 hbuf[UNR][8];
+            if (EPI == EPI_ADDNORM) {
+#pragma unroll
+                for (int u = 0; u < 3; ++u)
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) hbuf[u % UNR][v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (row < M) {
+#pragma unroll
+                    for (int u = 0; u < 3; ++u)
+                        if (u * 32 < BN) {
+                            const float4* hp = reinterpret_cast<const float4*>(g.C + (size_t)row * N + n0 + u * 32);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v) hbuf[u % UNR][v] = hp[v];
+                        }
+                }
+            }
             if (!mbar_wait(accf0 + 8 * buf, aph, abort_flag, g.acc_wait_ns ? g.acc_wait_ns : 1000000000ull)) {
                 if (lane == 0) {
                     raise_abort<PAIR>(abort_flag, rank);
@@ -447,8 +503,6 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int row = m0 + quarter * 32 + lane;
-            const uint32_t tbase = tmem_base + buf * BN + ((uint32_t)(quarter * 32) << 16);
 
             RowDst rd;
             rd.valid = row < M;
@@ -479,10 +533,89 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                 }
             }
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int cg = 0; cg < BN; cg += 32 * UNR) {
+              float ssq4[UNR];  // ADDNORM: sums of squares of this group's chunks
+#pragma unroll
+              for (int u = 0; u < UNR; ++u) ssq4[u] = 0.f;
+#pragma unroll
+              for (int u = 0; u < UNR; ++u) {
+                const int c0 = cg + 32 * u;
+                if (c0 >= BN) continue;
                 uint32_t r[32];
                 tmem_ld32(tbase + (uint32_t)c0, r);
                 const int col = n0 + c0;
+                if (EPI == EPI_ADDNORM) {
+                    // this warp's staging: two buffers of (fp32 tile 4 KB, swizzled | bf16 tile 2 KB, dense)
+                    const uint32_t sb32 =
+                        staging + (uint32_t)(warp - 2) * (uint32_t)cfg::WARP_STAGING + (uint32_t)(nchunk++ & 1u) * 6144u;
+                    const uint32_t sb16 = sb32 + 4096u;
+                    float4 hcur[8];
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) hcur[v] = hbuf[u][v];
+                    if (c0 + 96 < BN && row < M) {  // the chunk three ahead takes the slot this chunk frees next
+                        const float4* hp = reinterpret_cast<const float4*>(g.C + (size_t)row * N + col + 96);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) hbuf[(u + 3) % UNR][v] = hp[v];
+                    }
+                    // new residual = old + acc (one fp32 addition per element, as the reduce-add form did)
+                    float ss = 0.f;
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const float x0 = hcur[v].x + __uint_as_float(r[4 * v]);
+                        const float x1 = hcur[v].y + __uint_as_float(r[4 * v + 1]);
+                        const float x2 = hcur[v].z + __uint_as_float(r[4 * v + 2]);
+                        const float x3 = hcur[v].w + __uint_as_float(r[4 * v + 3]);
+                        ss += x0 * x0;
+                        ss += x1 * x1;
+                        ss += x2 * x2;
+                        ss += x3 * x3;
+                        r[4 * v] = __float_as_uint(x0);
+                        r[4 * v + 1] = __float_as_uint(x1);
+                        r[4 * v + 2] = __float_as_uint(x2);
+                        r[4 * v + 3] = __float_as_uint(x3);
+                    }
+                    ssq4[u] = ss;
+                    // one bulk tensor store per tile (the pair is one bulk group: the buffer used two chunks ago is
+                    // free once at most one group is still reading); rows past the buffers' capacity are clipped
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const uint32_t addr = sb32 + (uint32_t)lane * 128u + (uint32_t)((v ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r[4 * v]),
+                                     "r"(r[4 * v + 1]), "r"(r[4 * v + 2]), "r"(r[4 * v + 3])
+                                     : "memory");
+                    }
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        const uint32_t p0 = pack_bf16x2(__uint_as_float(r[8 * v]), __uint_as_float(r[8 * v + 1]));
+                        const uint32_t p1 = pack_bf16x2(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]));
+                        const uint32_t p2 = pack_bf16x2(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]));
+                        const uint32_t p3 = pack_bf16x2(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]));
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(sb16 + (uint32_t)lane * 64u +
+                                                                                    (uint32_t)v * 16u),
+                                     "r"(p0), "r"(p1), "r"(p2), "r"(p3)
+                                     : "memory");
+                    }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0 && m0 + quarter * 32 < M) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                                         &map_c),
+                                     "r"(col), "r"(m0 + quarter * 32), "r"(sb32)
+                                     : "memory");
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(
+                                         &map_hb),
+                                     "r"(col), "r"(m0 + quarter * 32), "r"(sb16)
+                                     : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    continue;
+                }
+                if (EPI == EPI_STORE && g.ssq_in != nullptr) {
+#pragma unroll
+                    for (int v = 0; v < 32; ++v) r[v] = __float_as_uint(__uint_as_float(r[v]) * rscale);
+                }
                 if (EPI == EPI_STORE || EPI == EPI_ADD) {
                     // registers -> swizzled staging tile (32 rows x 128 bytes) -> one TMA store / reduce-add
                     // of the 32 x 32 block; rows past M are clipped by the tensor map
@@ -522,8 +655,8 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     uint32_t o[8];
 #pragma unroll
                     for (int v = 0; v < 8; ++v) {
-                        const float g0 = __uint_as_float(r[4 * v]), u0 = __uint_as_float(r[4 * v + 1]);
-                        const float g1 = __uint_as_float(r[4 * v + 2]), u1 = __uint_as_float(r[4 * v + 3]);
+                        const float g0 = __uint_as_float(r[4 * v]) * rscale, u0 = __uint_as_float(r[4 * v + 1]) * rscale;
+                        const float g1 = __uint_as_float(r[4 * v + 2]) * rscale, u1 = __uint_as_float(r[4 * v + 3]) * rscale;
                         // silu(g) * u with ex2.approx and rcp.approx (about 1e-6 relative, far below bf16)
                         o[v] = pack_bf16x2(__fdividef(g0, 1.0f + __expf(-g0)) * u0,
                                            __fdividef(g1, 1.0f + __expf(-g1)) * u1);
@@ -541,15 +674,15 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
                             const float4 t = hi ? rope_hi[v] : rope_lo[v];  // cos, sin of pairs 2v and 2v+1
-                            const float a0 = __uint_as_float(r[4 * v]), b0 = __uint_as_float(r[4 * v + 1]);
-                            const float a1 = __uint_as_float(r[4 * v + 2]), b1 = __uint_as_float(r[4 * v + 3]);
+                            const float a0 = __uint_as_float(r[4 * v]) * rscale, b0 = __uint_as_float(r[4 * v + 1]) * rscale;
+                            const float a1 = __uint_as_float(r[4 * v + 2]) * rscale, b1 = __uint_as_float(r[4 * v + 3]) * rscale;
                             o[2 * v] = pack_bf16x2(a0 * t.x - b0 * t.y, a0 * t.y + b0 * t.x);
                             o[2 * v + 1] = pack_bf16x2(a1 * t.z - b1 * t.w, a1 * t.w + b1 * t.z);
                         }
                     } else {
 #pragma unroll
                         for (int v = 0; v < 16; ++v)
-                            o[v] = pack_bf16x2(__uint_as_float(r[2 * v]), __uint_as_float(r[2 * v + 1]));
+                            o[v] = pack_bf16x2(__uint_as_float(r[2 * v]) * rscale, __uint_as_float(r[2 * v + 1]) * rscale);
                     }
                     bf16* base = sec == 0 ? g.out + (size_t)row * D + cs
                                           : (bf16*)(sec == 1 ? g.kv.k : g.kv.v) + rd.kvoff + cs;
@@ -557,6 +690,17 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
 #pragma unroll
                     for (int v = 0; v < 4; ++v) dst[v] = make_uint4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
                 }
+              }
+              if (EPI == EPI_ADDNORM && row < M) {  // the group's partial sums: 16 contiguous bytes per row
+                  float* sp = g.ssq_out + (size_t)row * (N / 32) + (n0 + cg) / 32;
+                  if (BN >= 128) {
+                      *reinterpret_cast<float4*>(sp) = make_float4(ssq4[0], ssq4[1 % UNR], ssq4[2 % UNR], ssq4[3 % UNR]);
+                  } else {
+#pragma unroll
+                      for (int u = 0; u < UNR; ++u)
+                          if (u * 32 < BN) sp[u] = ssq4[u];
+                  }
+              }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -676,45 +820,60 @@ bool encode_map_c(CUtensorMap* map, const void* base, int rows, int N, int) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// bf16 row-major [rows, N] output, box = 32 columns (64 bytes) x 32 rows, no swizzle (dense 2 KB tile).
+bool encode_map_hb(CUtensorMap* map, const void* base, int rows, int N, int) {
+    EncodeFn enc = get_encode();
+    if (!enc) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)N * 2};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool make_map_c(CUtensorMap* map, const float* base, int rows, int N) {
     return cached_map(map, MapKey{base, rows, N, 32, 1}, encode_map_c);
 }
 
 template <int BN, int EPI>
-cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
-                   cudaStream_t s) {
+cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const CUtensorMap& mh,
+                   const GemmArgs& g, cudaStream_t s) {
     static int configured[64] = {0};
-    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<BN, EPI, false>, Cfg<BN>::SMEM, configured);
+    using cfg = Cfg<BN, false, EPI == EPI_ADDNORM>;
+    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<BN, EPI, false>, cfg::SMEM, configured);
     if (e0 != cudaSuccess) return e0;
     const int tiles = (g.N / BN) * ((g.M + BM - 1) / BM);
     const int grid = tiles < num_sms() ? tiles : num_sms();
-    return launch_k(k_gemm_tcgen05<BN, EPI, false>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<BN>::SMEM, s, ma, mw,
-                    mc, g);
+    return launch_k(k_gemm_tcgen05<BN, EPI, false>, dim3(grid), dim3(NUM_THREADS), (size_t)cfg::SMEM, s, ma, mw,
+                    mc, mh, g);
 }
 
 // CTA pairs: 256 x 256 tiles, one cluster of two CTAs per pair of SMs.
 template <int EPI>
-cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
-                        cudaStream_t s) {
+cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const CUtensorMap& mh,
+                        const GemmArgs& g, cudaStream_t s) {
     static int configured[64] = {0};
-    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<256, EPI, true>, Cfg<256, true>::SMEM, configured);
+    using cfg = Cfg<256, true, EPI == EPI_ADDNORM>;
+    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<256, EPI, true>, cfg::SMEM, configured);
     if (e0 != cudaSuccess) return e0;
     const int tiles = (g.N / 256) * ((g.M + 2 * BM - 1) / (2 * BM));
     const int pairs = num_sms() / 2;
     const int grid = 2 * (tiles < pairs ? tiles : pairs);
-    return launch_kc(k_gemm_tcgen05<256, EPI, true>, dim3(grid), dim3(NUM_THREADS), (size_t)Cfg<256, true>::SMEM, s, 2,
-                     ma, mw, mc, g);
+    return launch_kc(k_gemm_tcgen05<256, EPI, true>, dim3(grid), dim3(NUM_THREADS), (size_t)cfg::SMEM, s, 2,
+                     ma, mw, mc, mh, g);
 }
 
 template <int EPI>
-cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const GemmArgs& g,
-                      cudaStream_t s) {
+cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc,
+                      const CUtensorMap& mh, const GemmArgs& g, cudaStream_t s) {
     switch (bn) {
-        case 32: return launch<32, EPI>(ma, mw, mc, g, s);
-        case 64: return launch<64, EPI>(ma, mw, mc, g, s);
-        case 128: return launch<128, EPI>(ma, mw, mc, g, s);
-        case 512: return launch_pair<EPI>(ma, mw, mc, g, s);  // 256 x 256 on a CTA pair
-        default: return launch<256, EPI>(ma, mw, mc, g, s);
+        case 32: return launch<32, EPI>(ma, mw, mc, mh, g, s);
+        case 64: return launch<64, EPI>(ma, mw, mc, mh, g, s);
+        case 128: return launch<128, EPI>(ma, mw, mc, mh, g, s);
+        case 512: return launch_pair<EPI>(ma, mw, mc, mh, g, s);  // 256 x 256 on a CTA pair
+        default: return launch<256, EPI>(ma, mw, mc, mh, g, s);
     }
 }
 
@@ -742,11 +901,16 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
     }
     // large problems: 256 x 256 tiles on CTA pairs (a third less operand traffic per FLOP)
     const bool pair = !force_bn && bn == 256 && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2;
-    CUtensorMap ma, mw, mc;
+    CUtensorMap ma, mw, mc, mh;
     memset(&mc, 0, sizeof(mc));
+    memset(&mh, 0, sizeof(mh));
     const int map_rows = m_cap >= M ? m_cap : M;
-    if ((epi == EPI_STORE || epi == EPI_ADD) && !make_map_c(&mc, g.C, map_rows, N)) {
+    if ((epi == EPI_STORE || epi == EPI_ADD || epi == EPI_ADDNORM) && !make_map_c(&mc, g.C, map_rows, N)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed for the output (M=%d N=%d)", M, N);
+        return -3;
+    }
+    if (epi == EPI_ADDNORM && !cached_map(&mh, MapKey{g.hb, map_rows, N, 32, 2}, encode_map_hb)) {
+        snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed for the bf16 output (M=%d N=%d)", M, N);
         return -3;
     }
     if (!make_map(&ma, A, map_rows, K, BM) || !make_map(&mw, W, N, K, pair ? 128 : bn)) {
@@ -755,10 +919,11 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
     }
     cudaError_t e;
     switch (epi) {
-        case EPI_STORE: e = launch_bn<EPI_STORE>(pair ? 512 : bn, ma, mw, mc, g, s); break;
-        case EPI_ADD: e = launch_bn<EPI_ADD>(pair ? 512 : bn, ma, mw, mc, g, s); break;
-        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(pair ? 512 : bn, ma, mw, mc, g, s); break;
-        default: e = launch_bn<EPI_QKV>(pair ? 512 : bn, ma, mw, mc, g, s); break;
+        case EPI_STORE: e = launch_bn<EPI_STORE>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_ADD: e = launch_bn<EPI_ADD>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_ADDNORM: e = launch_bn<EPI_ADDNORM>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
+        default: e = launch_bn<EPI_QKV>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
     }
     if (e != cudaSuccess) {
         snprintf(err, errlen, "gemm launch: %s", cudaGetErrorString(e));
@@ -818,9 +983,50 @@ int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K
     return run(accumulate ? EPI_ADD : EPI_STORE, A, W, g, force_bn, 256, m_cap, s, err, errlen);
 }
 
-int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
-                        int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+namespace {
+void set_norm(GemmArgs& g, const NormIn& nin, int K) {
+    g.ssq_in = nin.ssq;
+    g.ssq_n = K / 32;
+    g.inv_dim = 1.0f / (float)K;
+    g.eps = nin.eps;
+}
+}  // namespace
+
+int gemm_tcgen05_head(const bf16* A, const bf16* W, float* C, int M, int N, int K, int m_cap, const NormIn& nin,
+                      int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
     GemmArgs g{};
+    g.C = C;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.error_flag = error_flag;
+    g.w_constant = 1;
+    set_norm(g, nin, K);
+    return run(EPI_STORE, A, W, g, 0, 256, m_cap, s, err, errlen);
+}
+
+int gemm_tcgen05_addnorm(const bf16* A, const bf16* W, float* h, bf16* hb, float* ssq_out, int M, int N, int K,
+                         int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+    if (((uintptr_t)h | (uintptr_t)hb) & 15) {
+        snprintf(err, errlen, "gemm: residual buffers must be 16-byte aligned");
+        return -1;
+    }
+    GemmArgs g{};
+    g.C = h;
+    g.hb = hb;
+    g.ssq_out = ssq_out;
+    g.M = M;
+    g.N = N;
+    g.K = K;
+    g.error_flag = error_flag;
+    g.w_constant = 1;
+    return run(EPI_ADDNORM, A, W, g, 0, 256, m_cap, s, err, errlen);
+}
+
+int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
+                        const NormIn& nin, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen) {
+    GemmArgs g{};
+    set_norm(g, nin, K);
     g.out = act;
     g.M = M;
     g.N = F2;
@@ -831,9 +1037,10 @@ int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, i
 }
 
 int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, int S, int layer,
-                     const float* rope_cs, const KvView& kv, int m_cap, int32_t* error_flag, cudaStream_t s,
-                     char* err, size_t errlen) {
+                     const float* rope_cs, const KvView& kv, int m_cap, const NormIn& nin, int32_t* error_flag,
+                     cudaStream_t s, char* err, size_t errlen) {
     GemmArgs g{};
+    set_norm(g, nin, st.D);
     g.out = q;
     g.M = st.nb * S * st.W;
     g.N = 3 * st.D;

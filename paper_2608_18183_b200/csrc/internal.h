@@ -54,8 +54,11 @@ struct AcceptArgs {
 
 // ---- row operations (model_kernels.cu)
 void launch_setup(const State& st, int phase /*0 round, 1 prefill*/, int compact, cudaStream_t s);
+// hb / ssq (bf16 model, may be null): the bf16 copy of the embedded rows and their partial sums of squares per
+// 32-column chunk, as the folded RMSNorm of the first projection wants them
 template <typename TA>
-void launch_embed(const State& st, int S, const TA* tok_emb, const TA* cls_emb, float* h, cudaStream_t s);
+void launch_embed(const State& st, int S, const TA* tok_emb, const TA* cls_emb, float* h, bf16* hb, float* ssq,
+                  cudaStream_t s);
 template <typename TA>
 void launch_rmsnorm(const float* h, const TA* gain, TA* out, int M, int D, float eps, cudaStream_t s);
 template <typename TA>
@@ -140,13 +143,26 @@ int gemm_tcgen05_run(const bf16* A, const bf16* W, float* C, int M, int N, int K
 int gemm_tcgen05_tile_n(int M, int N, int K);
 // Cached TMA descriptor of a row-major bf16 matrix [rows, cols]: box = 64 columns x box_rows rows, 128-byte swizzle.
 bool make_tensor_map_bf16(::CUtensorMap_st* map, const void* base, int rows, int cols, int box_rows);
+// RMSNorm folded around a GEMM: A holds the bf16 copy of the unnormalised residual rows x, W has the norm's gain
+// folded in, and the epilogue multiplies row m by rsqrt(sum(ssq[m][0 .. K/32)) / K + eps).  ssq null: no factor.
+struct NormIn {
+    const float* ssq;  // [M][K / 32] partial sums of squares of the fp32 rows
+    float eps;
+};
 // act[M, F] bf16 = silu(gate) * up, from A[M,K] . W13i^T where W13i[2F, K] holds gate row f at 2f, up row f at 2f+1.
 int gemm_tcgen05_swiglu(const bf16* A, const bf16* W13_interleaved, bf16* act, int M, int F2, int K, int m_cap,
-                        int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
+                        const NormIn& nin, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
+// logits[M, N] fp32 = norm(x) . W^T with the norm folded as above.
+int gemm_tcgen05_head(const bf16* A, const bf16* W, float* C, int M, int N, int K, int m_cap, const NormIn& nin,
+                      int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
+// Residual update h[M, N] fp32 += A[M,K] . W^T, which also leaves what the next folded norm needs: hb = bf16(h)
+// and ssq_out[M][N / 32] = sums of squares of the new h over each 32-column chunk (fixed order, no atomics).
+int gemm_tcgen05_addnorm(const bf16* A, const bf16* W, float* h, bf16* hb, float* ssq_out, int M, int N, int K,
+                         int m_cap, int32_t* error_flag, cudaStream_t s, char* err, size_t errlen);
 // QKV projection of the normed activations A[M, D] with the 2D RoPE and the paged KV write fused:
 // q[M, D] bf16 rotated; rotated k and v stored at each row's (cache row, sequence index).
 int gemm_tcgen05_qkv(const bf16* A, const bf16* Wqkv, bf16* q, const State& st, int S, int layer,
-                     const float* rope_cs, const KvView& kv, int m_cap, int32_t* error_flag, cudaStream_t s,
-                     char* err, size_t errlen);
+                     const float* rope_cs, const KvView& kv, int m_cap, const NormIn& nin, int32_t* error_flag,
+                     cudaStream_t s, char* err, size_t errlen);
 
 }  // namespace hbsjd

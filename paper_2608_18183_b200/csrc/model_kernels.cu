@@ -100,9 +100,12 @@ __global__ void k_noop() {
 void launch_noop(cudaStream_t s) { launch_k(k_noop, dim3(1), dim3(32), 0, s); }
 
 // ------------------------------------------------------------------ embedding gather
+// hb / ssq (may be null): bf16 copy of the row and its sums of squares per 32-column chunk (what the RMSNorm
+// folded into the first projection reads).  Warp w of the block owns chunks w, w + 4, ...; lane l element l.
 template <typename TA>
-__global__ void k_embed(State st, int S, const TA* __restrict__ tok_emb, const TA* __restrict__ cls_emb,
-                        float* __restrict__ h) {
+__global__ void __launch_bounds__(128) k_embed(State st, int S, const TA* __restrict__ tok_emb,
+                                               const TA* __restrict__ cls_emb, float* __restrict__ h,
+                                               bf16* __restrict__ hb, float* __restrict__ ssq) {
     pdl_trigger();
     pdl_wait();
     const int row = blockIdx.x;
@@ -110,29 +113,40 @@ __global__ void k_embed(State st, int S, const TA* __restrict__ tok_emb, const T
     const int slot = (row / st.W) % S;
     const int br = row / (st.W * S);
     const int n = st.slot_n[slot];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     float* dst = h + (size_t)row * st.D;
-    if (i >= n) {
-        for (int e = threadIdx.x; e < st.D; e += blockDim.x) dst[e] = 0.f;
-        return;
+    const TA* src = nullptr;
+    if (i < n) {
+        const int img = st.slot_img[slot];
+        const int s = st.slot_c[slot] + i;
+        if (s == 0) {
+            const int cls = br ? st.C : st.label[img];
+            src = cls_emb + (size_t)cls * st.D;
+        } else {
+            src = tok_emb + (size_t)st.seq[(size_t)img * (st.T + 1) + s] * st.D;
+        }
     }
-    const int img = st.slot_img[slot];
-    const int s = st.slot_c[slot] + i;
-    const TA* src;
-    if (s == 0) {
-        const int cls = br ? st.C : st.label[img];
-        src = cls_emb + (size_t)cls * st.D;
-    } else {
-        src = tok_emb + (size_t)st.seq[(size_t)img * (st.T + 1) + s] * st.D;
+    for (int chunk = wid; chunk * 32 < st.D; chunk += 4) {
+        const int e = chunk * 32 + lane;
+        const float v = (src != nullptr && e < st.D) ? to_f<TA>(src[e]) : 0.f;
+        if (e < st.D) {
+            dst[e] = v;
+            if (hb != nullptr) hb[(size_t)row * st.D + e] = __float2bfloat16_rn(v);
+        }
+        if (ssq != nullptr) {
+            const float ss = warp_sum(v * v);
+            if (lane == 0) ssq[(size_t)row * (st.D / 32) + chunk] = ss;
+        }
     }
-    for (int e = threadIdx.x; e < st.D; e += blockDim.x) dst[e] = to_f<TA>(src[e]);
 }
 
 template <typename TA>
-void launch_embed(const State& st, int S, const TA* tok_emb, const TA* cls_emb, float* h, cudaStream_t s) {
-    launch_k(k_embed<TA>, dim3(st.nb * S * st.W), dim3(128), 0, s, st, S, tok_emb, cls_emb, h);
+void launch_embed(const State& st, int S, const TA* tok_emb, const TA* cls_emb, float* h, bf16* hb, float* ssq,
+                  cudaStream_t s) {
+    launch_k(k_embed<TA>, dim3(st.nb * S * st.W), dim3(128), 0, s, st, S, tok_emb, cls_emb, h, hb, ssq);
 }
-template void launch_embed<float>(const State&, int, const float*, const float*, float*, cudaStream_t);
-template void launch_embed<bf16>(const State&, int, const bf16*, const bf16*, float*, cudaStream_t);
+template void launch_embed<float>(const State&, int, const float*, const float*, float*, bf16*, float*, cudaStream_t);
+template void launch_embed<bf16>(const State&, int, const bf16*, const bf16*, float*, bf16*, float*, cudaStream_t);
 
 // ------------------------------------------------------------------ RMSNorm: out = x * rsqrt(mean(x^2)+eps) * g
 // One warp per row; the row stays in registers between the two passes (D <= 2048 through the vector path).

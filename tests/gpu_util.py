@@ -42,10 +42,11 @@ def bf16_logit_tol(sigma, n_layers):
     return std, max(2e-2, 5.5 * std)
 
 
-def noise_floor(model, w, toks_row, label, c):
+def noise_floor(model, w, toks_row, label, c, norm_folded=False):
     """Logit noise floor of bf16 activations at one window: the oracle against ITSELF in its diagnostic form --
-    every dot product accumulated in fp32 instead of double, and the attention weights rounded to bf16 before they
-    multiply the values (the tensor-core formulation of attention); nothing else changed -- on sequence indices
+    every dot product accumulated in fp32 instead of double, the attention weights rounded to bf16 before they
+    multiply the values (the tensor-core formulation of attention) and, for contexts that fold RMSNorm into their
+    GEMMs, the norm's row factor applied after the projection; nothing else changed -- on sequence indices
     c .. c+n-1 after pre-filling 0 .. c-1.  A difference of one ulp anywhere flips bf16 roundings downstream,
     after which the two runs differ at bf16-noise level; this measures how much of a logit that is at this
     depth and logit scale: what two correct bf16 implementations must be expected to differ by.  The
@@ -56,7 +57,7 @@ def noise_floor(model, w, toks_row, label, c):
     n = min(W, T - c)
     out = []
     for diag in (False, True):
-        model.set_diag(acc_f32=diag, attn_w_bf16=diag)
+        model.set_diag(acc_f32=diag, attn_w_bf16=diag, norm_folded=diag and norm_folded)
         try:
             cache = model.new_cache()
             for pc in range(0, c, W):
@@ -68,9 +69,9 @@ def noise_floor(model, w, toks_row, label, c):
     return float(d.max()), float(d.sum()), int(d.size), float(out[0].std())
 
 
-def floor_of(model, w, toks, lab, k, ids):
+def floor_of(model, w, toks, lab, k, ids, norm_folded=False):
     """Noise floor over the first windows of the images `ids`: (max, mean over all their logits)."""
-    fl = [noise_floor(model, w, toks[b], int(lab[b]), int(k[b])) for b in ids if k[b] < w.shape.T]
+    fl = [noise_floor(model, w, toks[b], int(lab[b]), int(k[b]), norm_folded) for b in ids if k[b] < w.shape.T]
     return max(f[0] for f in fl), sum(f[1] for f in fl) / sum(f[2] for f in fl)
 
 
@@ -168,7 +169,7 @@ def lockstep(ctx, model, w, toks, k, lab, seed, greedy=False, image_ids=None, ma
             if floor_every_round:
                 both = []
                 for diag in (False, True):
-                    model.set_diag(acc_f32=diag, attn_w_bf16=diag)
+                    model.set_diag(acc_f32=diag, attn_w_bf16=diag, norm_folded=diag and ctx.fold_norm)
                     try:
                         both.append(model.forward_full(int(lab[b]), o_seq[x][:c + n])[c:].astype(np.float64))
                     finally:

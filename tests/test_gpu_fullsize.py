@@ -60,8 +60,8 @@ def test_fullsize_properties(big):
     assert not np.array_equal(other.cpu().numpy(), ref)
 
 
-def _check_against_floor(rep, model, w, toks, lab, k, ids, label):
-    floor_max, floor_mean = G.floor_of(model, w, toks, lab, k, ids)
+def _check_against_floor(ctx, rep, model, w, toks, lab, k, ids, label):
+    floor_max, floor_mean = G.floor_of(model, w, toks, lab, k, ids, norm_folded=ctx.fold_norm)
     G.check_logits_against_floor(rep, floor_max, floor_mean, label)
     assert rep["max_p_err"] <= 1e-6
     G.check_flips_explained(rep)
@@ -76,7 +76,7 @@ def test_fullsize_sampled_images_in_lockstep_with_the_oracle(big):
     model = O.Model(w.shape, weights)
     rep = G.lockstep(ctx, model, w, toks, k, lab, 23, image_ids=ids, max_rounds=4, park_others=False)
     assert rep["tokens"] >= 4 * len(ids)
-    _check_against_floor(rep, model, w, toks, lab, k, ids, f"{w.name} ids {ids} k {[int(k[b]) for b in ids]}")
+    _check_against_floor(ctx, rep, model, w, toks, lab, k, ids, f"{w.name} ids {ids} k {[int(k[b]) for b in ids]}")
 
 
 def test_fullsize_one_image_to_completion(big):
@@ -91,4 +91,4 @@ def test_fullsize_one_image_to_completion(big):
     model = O.Model(w.shape, weights)
     rep = G.lockstep(ctx, model, w, toks, k2, lab, 29, image_ids=[b], park_others=False)
     assert rep["tokens"] == 40
-    _check_against_floor(rep, model, w, toks, lab, k2, [b], f"{w.name} image {b} to completion")
+    _check_against_floor(ctx, rep, model, w, toks, lab, k2, [b], f"{w.name} image {b} to completion")
