@@ -296,6 +296,13 @@ def main():
             "frac_of_measured_burst": gemm_tflops / pk["bf16_tflops"],
             "frac_of_nominal": gemm_tflops / NOMINAL_PEAKS["bf16_tflops"],
             "nominal_peak": NOMINAL_PEAKS["bf16_tflops"]}
+    # the same class split by the activation rows of the launch: full rounds against the thinning tail of a rollout
+    roof["by_rows"] = {
+        name: {"launches": b["launches"], "ms_per_step": b["ms"] / args.steps,
+               "achieved": b["work"] / (b["ms"] * 1e-3) / 1e12 if b["ms"] > 0 else 0.0,
+               "frac": b["work"] / (b["ms"] * 1e-3) / 1e12 / pk["bf16_tflops_sustained"] if b["ms"] > 0 else 0.0,
+               "frac_net_of_launch_floor": net(b) / 1e12 / pk["bf16_tflops_sustained"]}
+        for name, b in prof["gemm_by_rows"].items()}
     if w.shape.dtype != "bf16":
         roof.update(bound="alu", peak=72.0, peak_source="fp32 CUDA-core FMA: 148 SMs x 128 lanes x 2 x 1.9 GHz")
         roof["frac"] = gemm_tflops / 72.0

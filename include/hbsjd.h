@@ -204,9 +204,12 @@ int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int 
  * epilogue warps on their accumulator shortened to that many nanoseconds (Sec. 4.2 verifier forward; the paper has
  * no counterpart of the failure path).  A limit shorter than the main loop makes a healthy pipeline take the
  * time-out path: every role leaves its loop, copies and MMAs in flight are drained, TMEM is freed, the call
- * returns HBSJD_ETIMEOUT with C partly written, and the context stays usable.  Tests use it to exercise that path. */
+ * returns HBSJD_ETIMEOUT with C partly written, and the context stays usable.  Tests use it to exercise that path.
+ * tile (bf16 contexts, accumulate 0 or 1): 0 = the library's own choice for the shape; 32, 64, 128, 256 = one CTA
+ * per 128 x tile block of C; 512 = 256 x 256 blocks on CTA pairs (N a multiple of 256).  Every choice gives the
+ * same bits (each element's products are summed in the same order); HBSJD_EINVAL for any other value. */
 int hbsjd_debug_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate,
-                     int reps, unsigned int acc_wait_ns);
+                     int reps, unsigned int acc_wait_ns, int tile);
 
 /* Chooses the form of RMSNorm of a bf16 context (Sec. 4.2 verifier forward; the paper does not go below the model):
  * on = 1 folds it into the GEMM epilogues (bf16 copy of the unnormalised residual stream as the operand, gain in the
@@ -314,6 +317,11 @@ typedef struct {
     double work[4];
     int64_t launches[4];
     int64_t dropped;   /* launches not timed because the event pool was exhausted */
+    /* the GEMM class again, split by the number of activation rows M of the launch:
+     * M <= 512, 512 < M <= 2048, 2048 < M <= 6144, M > 6144 */
+    double gemm_ms_by_rows[4];
+    double gemm_work_by_rows[4];
+    int64_t gemm_launches_by_rows[4];
 } hbsjd_kernel_profile;
 int hbsjd_profile(hbsjd_ctx *c, int enable);
 int hbsjd_profile_read(hbsjd_ctx *c, hbsjd_kernel_profile *out);

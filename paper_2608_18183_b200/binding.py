@@ -47,10 +47,12 @@ class hbsjd_stats(C.Structure):
 
 class hbsjd_kernel_profile(C.Structure):
     _fields_ = [("ms", C.c_double * 4), ("work", C.c_double * 4), ("launches", C.c_int64 * 4),
-                ("dropped", C.c_int64)]
+                ("dropped", C.c_int64), ("gemm_ms_by_rows", C.c_double * 4), ("gemm_work_by_rows", C.c_double * 4),
+                ("gemm_launches_by_rows", C.c_int64 * 4)]
 
 
 PROF_CLASSES = ("gemm", "attention", "accept", "other")
+PROF_GEMM_ROW_BINS = ("rows<=512", "rows<=2048", "rows<=6144", "rows>6144")
 
 
 class hbsjd_verify_desc(C.Structure):
@@ -102,7 +104,7 @@ def load():
         L.hbsjd_debug_read.argtypes = [vp, C.c_int, C.c_int, vp, C.c_size_t]
         L.hbsjd_debug_forward.argtypes = [vp, C.c_int, C.c_int]
         L.hbsjd_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int]
-        L.hbsjd_debug_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint]
+        L.hbsjd_debug_gemm.argtypes = [vp, vp, vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_uint, C.c_int]
         L.hbsjd_debug_shuffle_pages.argtypes = [vp, C.c_uint64]
         L.hbsjd_debug_fold_norm.argtypes = [vp, C.c_int]
         L.hbsjd_bikl.argtypes = [vp, vp, vp, C.c_int, vp]
@@ -201,7 +203,9 @@ class Context:
         p = hbsjd_kernel_profile()
         self._check(self.lib.hbsjd_profile_read(self.h, C.byref(p)), "hbsjd_profile_read")
         return {n: dict(ms=p.ms[i], work=p.work[i], launches=p.launches[i]) for i, n in enumerate(PROF_CLASSES)} | {
-            "dropped": p.dropped}
+            "dropped": p.dropped,
+            "gemm_by_rows": {n: dict(ms=p.gemm_ms_by_rows[i], work=p.gemm_work_by_rows[i],
+                                     launches=p.gemm_launches_by_rows[i]) for i, n in enumerate(PROF_GEMM_ROW_BINS)}}
 
     def hbsjd_profile_launch_floor(self, reps=200) -> float:
         """Median event bracket of an empty kernel launch, microseconds."""
@@ -296,13 +300,13 @@ class Context:
                                         1 if accumulate else 0), "hbsjd_gemm")
         return Cout
 
-    def hbsjd_debug_gemm(self, A, W, Cout, accumulate=False, reps=1, acc_wait_ns=0):
+    def hbsjd_debug_gemm(self, A, W, Cout, accumulate=False, reps=1, acc_wait_ns=0, tile=0):
         """hbsjd_gemm `reps` times back to back; acc_wait_ns > 0 shortens the epilogue's bounded wait (time-out test)."""
         M, K = A.shape
         N = W.shape[0]
         assert W.shape[1] == K and tuple(Cout.shape) == (M, N) and Cout.dtype == self._torch.float32
         self._check(self.lib.hbsjd_debug_gemm(self.h, A.data_ptr(), W.data_ptr(), Cout.data_ptr(), M, N, K,
-                                              int(accumulate), reps, acc_wait_ns), "hbsjd_debug_gemm")
+                                              int(accumulate), reps, acc_wait_ns, tile), "hbsjd_debug_gemm")
         return Cout
 
     def hbsjd_debug_fold_norm(self, on: bool):

@@ -65,7 +65,7 @@ struct hbsjd_ctx {
     int32_t* m_sync;                              // [1] smallest commit of the round (batch-synchronous progress)
     // per-class event timing
     bool profiling;
-    struct ProfSlot { cudaEvent_t a, b; int cls; double work; };
+    struct ProfSlot { cudaEvent_t a, b; int cls; double work; int rows; };
     std::vector<ProfSlot> pool;
     int pool_used;
     int pending_attn;  // attention launches of the current forward whose byte count waits for the counters
@@ -87,7 +87,7 @@ namespace {
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 // Brackets the launches issued between prof_begin and prof_end with an event pair of class `cls`.
-int prof_begin(hbsjd_ctx* c, int cls, double work) {
+int prof_begin(hbsjd_ctx* c, int cls, double work, int rows = 0) {
     if (!c->profiling) return -1;
     if (c->pool_used >= (int)c->pool.size()) {
         c->prof.dropped++;
@@ -96,6 +96,7 @@ int prof_begin(hbsjd_ctx* c, int cls, double work) {
     hbsjd_ctx::ProfSlot& s = c->pool[c->pool_used];
     s.cls = cls;
     s.work = work;
+    s.rows = rows;
     cudaEventRecord(s.a, c->stream);
     return c->pool_used++;
 }
@@ -115,6 +116,12 @@ void prof_resolve(hbsjd_ctx* c, double attn_bytes, double accept_bytes) {
         c->prof.ms[s.cls] += ms;
         c->prof.work[s.cls] += work;
         c->prof.launches[s.cls] += 1;
+        if (s.cls == HBSJD_PROF_GEMM && s.rows > 0) {
+            const int bin = s.rows <= 512 ? 0 : s.rows <= 2048 ? 1 : s.rows <= 6144 ? 2 : 3;
+            c->prof.gemm_ms_by_rows[bin] += ms;
+            c->prof.gemm_work_by_rows[bin] += work;
+            c->prof.gemm_launches_by_rows[bin] += 1;
+        }
     }
     c->pool_used = 0;
 }
@@ -143,12 +150,12 @@ KvView kv_view(const hbsjd_ctx* c) {
 // w_constant: W is one of the model's weight matrices (see gemm_tcgen05_run)
 template <typename TA>
 int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int m_cap = 0,
-         int w_constant = 1, unsigned int acc_wait_ns = 0);
+         int w_constant = 1, unsigned int acc_wait_ns = 0, int tile = 0);
 
 template <>
 int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int, int,
-                unsigned int) {
-    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
+                unsigned int, int) {
+    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K, M);
     launch_gemm_simt<float>((const float*)A, (const float*)W, C, M, N, K, accumulate, c->stream);
     prof_end(c, ps);
     c->launches++;
@@ -157,10 +164,10 @@ int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int
 
 template <>
 int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
-               int m_cap, int w_constant, unsigned int acc_wait_ns) {
+               int m_cap, int w_constant, unsigned int acc_wait_ns, int tile) {
     c->launches++;
-    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K);
-    const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, 0, m_cap,
+    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K, M);
+    const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, tile, m_cap,
                                     c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err), w_constant,
                                     acc_wait_ns);
     prof_end(c, ps);
@@ -254,7 +261,7 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
     };
     // residual update h += A W^T
     auto residual = [&](const void* A, const void* W, int K) {
-        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * D * K);
+        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * D * K, M);
         int rc;
         if (fold)
             rc = gemm_tcgen05_addnorm((const bf16*)A, (const bf16*)W, c->h, a, c->ssq, M, D, K, Mcap, eflag, s, c->err,
@@ -273,7 +280,7 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
         const LayerW& w = c->layers[l];
         int rc, ps;
         if (!fold) norm(w.g_attn);
-        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D);
+        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D, M);
         rc = gemm_tcgen05_qkv(a, (const bf16*)w.w_qkv, (bf16*)c->q, st, S, l, c->rope_cs, kv, Mcap, nin, eflag, s,
                               c->err, sizeof(c->err));
         prof_end(c, ps);
@@ -291,7 +298,7 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
         if ((rc = residual(c->o, w.w_o, D))) return done(rc);
         if (l == stop_layer && stop_stage == 0) return 0;
         if (!fold) norm(w.g_ffn);
-        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D);
+        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D, M);
         rc = gemm_tcgen05_swiglu(a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D, Mcap, nin, eflag, s, c->err,
                                  sizeof(c->err));
         prof_end(c, ps);
@@ -302,7 +309,7 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
     }
     if (want_logits) {
         if (!fold) norm(c->g_out);
-        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * st.V * D);
+        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * st.V * D, M);
         const int rc = gemm_tcgen05_head(a, (const bf16*)c->w_head, c->logits, M, st.V, D, Mcap, nin, eflag, s,
                                          c->err, sizeof(c->err));
         prof_end(c, ps);
@@ -1220,11 +1227,11 @@ int hbsjd_debug_read(hbsjd_ctx* c, int what, int index, void* host_dst, size_t m
 }
 
 int hbsjd_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate) {
-    return hbsjd_debug_gemm(c, A, W, C, M, N, K, accumulate, 1, 0);
+    return hbsjd_debug_gemm(c, A, W, C, M, N, K, accumulate, 1, 0, 0);
 }
 
 int hbsjd_debug_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
-                     int reps, unsigned int acc_wait_ns) {
+                     int reps, unsigned int acc_wait_ns, int tile) {
     if (!c || !A || !W || !C || M < 1 || N < 1 || K < 1 || reps < 1) return HBSJD_EINVAL;
     if (accumulate == 2 && (!c->bf16_model || N != c->d.dim || M > 2 * c->Bmax * c->Wmax)) {
         snprintf(c->err, sizeof(c->err), "hbsjd_debug_gemm: the residual-update form needs a bf16 context, N = dim and "
@@ -1242,7 +1249,7 @@ int hbsjd_debug_gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M
             if (rc) rc = rc == -1 ? HBSJD_EINVAL : HBSJD_ECUDA;
         } else {
             // W is the caller's buffer, possibly written by earlier work of the stream: no early fetch of its tiles
-            rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate, 0, 0, acc_wait_ns)
+            rc = c->bf16_model ? gemm<bf16>(c, A, W, C, M, N, K, accumulate, 0, 0, acc_wait_ns, tile)
                                : gemm<float>(c, A, W, C, M, N, K, accumulate);
         }
         if (rc) return rc;

@@ -248,6 +248,15 @@ __global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __g
                     qa[kc][3] = *reinterpret_cast<const uint32_t*>(qrow1 + d + 8);
                 }
             }
+            {   // the next item's query rows towards L1 while this item's keys stream (one 128-byte line per row)
+                const int pos2 = (stripe + 1) * grid < n_items ? position(stripe + 1) : n_items;
+                Item nx;
+                if (lane < 16 && pos2 < n_items && item_at(a, s_tab, pos2, nx)) {
+                    const bf16* nq = a.q + ((size_t)nx.prow * st.W + min(wq * 16 + lane, st.W - 1)) * st.D +
+                                     (nx.head0 + wh) * DH;
+                    asm volatile("prefetch.global.L1 [%0];" ::"l"(nq));
+                }
+            }
             const bool warp_active = wq * 16 < n;  // q-blocks wholly past the window only keep the ring moving
             const int s0 = c + i0, s1 = c + i1;    // sequence index of this thread's two query rows
             float o[8][4];

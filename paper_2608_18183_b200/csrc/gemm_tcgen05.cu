@@ -889,10 +889,12 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
                  M, N, K);
         return -1;
     }
-    if (force_bn != 0 && force_bn != 32 && force_bn != 64 && force_bn != 128 && force_bn != 256) {
-        snprintf(err, errlen, "gemm: tile width %d is not one of 32, 64, 128, 256", force_bn);
+    if (force_bn != 0 && force_bn != 32 && force_bn != 64 && force_bn != 128 && force_bn != 256 && force_bn != 512) {
+        snprintf(err, errlen, "gemm: tile %d is not one of 32, 64, 128, 256 (one CTA) or 512 (CTA pair)", force_bn);
         return -1;
     }
+    const bool force_pair = force_bn == 512;
+    if (force_pair) force_bn = 256;
     int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N, K);
     while (bn > max_bn) bn >>= 1;
     if (bn < 32 || N % bn != 0) {
@@ -900,7 +902,7 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
         return -1;
     }
     // large problems: 256 x 256 tiles on CTA pairs (a third less operand traffic per FLOP)
-    const bool pair = !force_bn && bn == 256 && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2;
+    const bool pair = bn == 256 && (force_pair || (!force_bn && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2));
     CUtensorMap ma, mw, mc, mh;
     memset(&mc, 0, sizeof(mc));
     memset(&mh, 0, sizeof(mh));
