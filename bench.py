@@ -97,11 +97,11 @@ def oracle_sample(w, weights, toks, k, lab, seed, ids, n_rounds):
 
 
 def sample_plan(w, k):
-    """Bounded oracle sample per workload: (image ids, rounds, description), sized for roughly 5-30 s of CPU
+    """Bounded oracle sample per workload: (image ids, rounds, description), sized for roughly 10-15 s of CPU
     work per step.  The large models take the images with the shortest prefixes (cheapest pre-filling)."""
     order = [int(i) for i in np.argsort(k, kind="stable")]
-    n_img, n_rounds = {"tiny": (w.batch, 0), "tiny_bf16": (w.batch, 0), "small_bf16": (w.batch, 0), "B": (8, 6),
-                       "L": (2, 4), "XL": (1, 3), "stress": (2, 4)}.get(w.name, (1, 1))
+    n_img, n_rounds = {"tiny": (w.batch, 0), "tiny_bf16": (w.batch, 0), "small_bf16": (w.batch, 0), "B": (8, 16),
+                       "L": (2, 8), "XL": (1, 6), "stress": (2, 8)}.get(w.name, (1, 1))
     ids = list(range(n_img)) if n_img == w.batch else order[:n_img]
     what = (f"{n_img} image(s) of the batch with the shortest prefixes (ids {ids}, prefix lengths "
             f"{[int(k[i]) for i in ids]}): prefix pre-filling + {n_rounds or 'all'} rounds")

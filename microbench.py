@@ -3,6 +3,8 @@
     python microbench.py accept   # verification step at a paper-like commit length
     python microbench.py probs    # probability pipeline on 4096 rows
     python microbench.py gemm     # decoder GEMM shapes of a workload, each timed alone
+    python microbench.py gemm_tiles  # the same shapes with every tile shape forced, over --row-list
+    python microbench.py gemm_floor  # cost of a small GEMM launch with and without the host's launch rate in it
     python microbench.py bikl     # bidirectional-KL reduction (Eq. 3) on 4096 row pairs
     python microbench.py score    # teacher/student scoring of a batch of trajectories (Eq. 3)
     python microbench.py attention  # ragged attention at fixed context lengths (--workload L|XL, --contexts a,b,..)
@@ -177,6 +179,8 @@ def bench_gemm(args):
                             ("attention out (+=, bf16 copy, sums of squares)", D, D, 2), ("gate|up", 2 * F, D, 0),
                             ("down (+=)", D, F, 1), ("down (+=, bf16 copy, sums of squares)", D, F, 2),
                             ("head", V, D, 0)]:
+        if args.only and not name.startswith(args.only):
+            continue
         A = torch.randn(M, K, device="cuda", generator=g).bfloat16()
         Wt = (torch.randn(N, K, device="cuda", generator=g) * 0.05).bfloat16()
         Cm = torch.zeros(M, N, device="cuda")
@@ -185,6 +189,68 @@ def bench_gemm(args):
         us = _median_us(torch, burst, reps=5, warm=2) / 20
         print(json.dumps({"case": "gemm", "name": name, "M": M, "N": N, "K": K, "accumulate": acc,
                           "us": round(us, 1), "TFLOP_s": round(2.0 * M * N * K / us / 1e6, 1)}))
+    ctx.hbsjd_destroy()
+
+
+def _gemm_context(binding, synth, s, rows):
+    sh = synth.ModelShape(1, s.dim, s.n_heads, 64, 64, 4, 4, 3, "bf16")
+    return binding.Context(sh, synth.make_weights(sh, 3, target_entropy=None), (rows + 63) // 64, 32)
+
+
+def bench_gemm_tiles(args):
+    """Every tile shape of the GEMM kernel on the decoder's shapes, over a range of activation rows M."""
+    import torch
+    from paper_2608_18183_b200 import binding, synth
+    s = synth.WORKLOADS[args.workload].shape
+    D, F, V = s.dim, s.ffn_hidden, s.vocab
+    ms = [int(x) for x in args.row_list.split(",")]
+    ctx = _gemm_context(binding, synth, s, max(ms))
+    g = torch.Generator(device="cuda")
+    g.manual_seed(args.seed)
+    for name, N, K, acc in [("qkv", 3 * D, D, 0), ("attention out (+=)", D, D, 1), ("gate|up", 2 * F, D, 0),
+                            ("down (+=)", D, F, 1), ("head", V, D, 0)]:
+        Wt = (torch.randn(N, K, device="cuda", generator=g) * 0.05).bfloat16()
+        for M in ms:
+            A = torch.randn(M, K, device="cuda", generator=g).bfloat16()
+            Cm = torch.zeros(M, N, device="cuda")
+            us = {}
+            for tile in (0, 32, 64, 128, 256, 512):  # 0: the library's choice; 512: 256 x 256 on CTA pairs
+                if tile and N % min(tile, 256):
+                    continue
+                def burst():
+                    ctx.hbsjd_debug_gemm(A, Wt, Cm, accumulate=acc, reps=20, tile=tile)
+                us[str(tile)] = round(_median_us(torch, burst, reps=5, warm=2) / 20, 1)
+            print(json.dumps({"case": "gemm_tiles", "name": name, "M": M, "N": N, "K": K, "us_by_tile": us}))
+    ctx.hbsjd_destroy()
+
+
+def bench_gemm_floor(args):
+    """What a GEMM launch costs however small it is: 800 launches queued behind a spin of about 10 ms, so that the
+    host's launch rate is outside the figure (and the same without the spin, where it is inside)."""
+    import time
+    import torch
+    from paper_2608_18183_b200 import binding, synth
+    s = synth.WORKLOADS[args.workload].shape
+    ctx = _gemm_context(binding, synth, s, 256)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(args.seed)
+    for M, N, K in ((256, s.dim, 64), (256, s.dim, s.dim), (256, 3 * s.dim, s.dim), (64, s.dim, s.ffn_hidden)):
+        A = torch.randn(M, K, device="cuda", generator=g).bfloat16()
+        Wt = (torch.randn(N, K, device="cuda", generator=g) * 0.05).bfloat16()
+        Cm = torch.zeros(M, N, device="cuda")
+        ctx.hbsjd_debug_gemm(A, Wt, Cm, reps=50)
+        out = {}
+        for label, spin in (("host_in_figure", 0), ("queued_behind_spin", 20_000_000)):
+            torch.cuda.synchronize()
+            e1, e2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if spin:
+                torch.cuda._sleep(spin)
+            e1.record()
+            ctx.hbsjd_debug_gemm(A, Wt, Cm, reps=800)
+            e2.record()
+            torch.cuda.synchronize()
+            out[label] = round(e1.elapsed_time(e2) * 1e3 / 800, 2)
+        print(json.dumps({"case": "gemm_floor", "M": M, "N": N, "K": K, "us_per_launch": out}))
     ctx.hbsjd_destroy()
 
 
@@ -292,7 +358,8 @@ def bench_attention(args):
 
 def main(argv=None):
     ap = argparse.ArgumentParser(description=__doc__.split("\n")[0])
-    ap.add_argument("case", choices=["accept", "probs", "gemm", "bikl", "score", "attention"])
+    ap.add_argument("case", choices=["accept", "probs", "gemm", "gemm_tiles", "gemm_floor", "bikl", "score",
+                                     "attention"])
     ap.add_argument("--contexts", default="0,32,64,128,192,223")
     ap.add_argument("--workload", default="L")
     ap.add_argument("--batch", type=int, default=0)
@@ -302,11 +369,13 @@ def main(argv=None):
     ap.add_argument("--cfg-scale", type=float, default=4.0)
     ap.add_argument("--target-commit", type=float, default=2.3)
     ap.add_argument("--rows", type=int, default=0)
+    ap.add_argument("--row-list", default="512,2048,4096,5120,8192", help="gemm_tiles: activation row counts")
+    ap.add_argument("--only", default="", help="gemm: only the shapes whose name starts with this")
     ap.add_argument("--seed", type=int, default=1)
     args = ap.parse_args(argv)
     if args.case in ("probs", "bikl") and not args.rows:
         args.rows = 4096
-    {"accept": bench_accept, "probs": bench_probs, "gemm": bench_gemm, "bikl": bench_bikl,
+    {"accept": bench_accept, "probs": bench_probs, "gemm": bench_gemm, "gemm_tiles": bench_gemm_tiles, "gemm_floor": bench_gemm_floor, "bikl": bench_bikl,
      "score": bench_score, "attention": bench_attention}[args.case](args)
 
 

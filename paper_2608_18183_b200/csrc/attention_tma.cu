@@ -135,7 +135,7 @@ __device__ __forceinline__ bool item_at(const AttnArgs& a, const int* s_tab, int
 }
 
 template <int QB>
-__global__ void __launch_bounds__((QB * HPC + 1) * 32) k_attention_tma(const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__((QB * HPC + 1) * 32, QB >= 3 ? 2 : 3) k_attention_tma(const __grid_constant__ CUtensorMap map_k,
                                                                        const __grid_constant__ CUtensorMap map_v,
                                                                        const AttnArgs a) {
     pdl_trigger();
@@ -394,10 +394,18 @@ cudaError_t launch_qb(const CUtensorMap& mk, const CUtensorMap& mv, const AttnAr
     static int configured[64] = {0};
     cudaError_t e = ensure_dynamic_smem(k_attention_tma<QB>, smem, configured);
     if (e != cudaSuccess) return e;
-    // resident CTAs per SM by shared memory (228 KB per SM, 1 KB reserved per CTA)
-    int per_sm = (228 * 1024) / (smem + 1024);
-    if (per_sm < 1) per_sm = 1;
-    if (per_sm > 3) per_sm = 3;
+    // resident CTAs per SM (registers and shared memory), at most 3: the grid is exactly what is resident at once
+    static int resident[64] = {0};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    dev &= 63;
+    if (resident[dev] == 0) {
+        int n = 0;
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k_attention_tma<QB>, threads, (size_t)smem);
+        if (e != cudaSuccess) return e;
+        resident[dev] = n < 1 ? 1 : (n > 3 ? 3 : n);
+    }
+    const int per_sm = resident[dev];
     const long items = (long)a.S * a.st.nb * a.G;
     long grid = (long)device_sm_count() * per_sm;
     if (grid > items) grid = items;
