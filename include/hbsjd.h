@@ -206,7 +206,7 @@ int hbsjd_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int 
  * time-out path: every role leaves its loop, copies and MMAs in flight are drained, TMEM is freed, the call
  * returns HBSJD_ETIMEOUT with C partly written, and the context stays usable.  Tests use it to exercise that path.
  * tile (bf16 contexts, accumulate 0 or 1): 0 = the library's own choice for the shape; 32, 64, 128, 256 = one CTA
- * per 128 x tile block of C; 512 = 256 x 256 blocks on CTA pairs (N a multiple of 256).  Every choice gives the
+ * per 128 x tile block of C; 512 / 640 = 256 x 256 / 256 x 128 blocks on CTA pairs (N a multiple of 256 / 128).  Every choice gives the
  * same bits (each element's products are summed in the same order); HBSJD_EINVAL for any other value. */
 int hbsjd_debug_gemm(hbsjd_ctx *c, const void *A, const void *W, float *C, int M, int N, int K, int accumulate,
                      int reps, unsigned int acc_wait_ns, int tile);

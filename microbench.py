@@ -214,8 +214,9 @@ def bench_gemm_tiles(args):
             A = torch.randn(M, K, device="cuda", generator=g).bfloat16()
             Cm = torch.zeros(M, N, device="cuda")
             us = {}
-            for tile in (0, 32, 64, 128, 256, 512):  # 0: the library's choice; 512: 256 x 256 on CTA pairs
-                if tile and N % min(tile, 256):
+            # 0: the library's choice; 512 / 640: 256 x 256 / 256 x 128 tiles on CTA pairs
+            for tile in (0, 32, 64, 128, 256, 512, 640):
+                if tile and N % (tile if tile < 512 else 768 - tile):
                     continue
                 def burst():
                     ctx.hbsjd_debug_gemm(A, Wt, Cm, accumulate=acc, reps=20, tile=tile)

@@ -850,18 +850,18 @@ cudaError_t launch(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorM
                     mc, mh, g);
 }
 
-// CTA pairs: 256 x 256 tiles, one cluster of two CTAs per pair of SMs.
-template <int EPI>
+// CTA pairs: 256 x BN tiles (BN = 256 or 128), one cluster of two CTAs per pair of SMs.
+template <int BN, int EPI>
 cudaError_t launch_pair(const CUtensorMap& ma, const CUtensorMap& mw, const CUtensorMap& mc, const CUtensorMap& mh,
                         const GemmArgs& g, cudaStream_t s) {
     static int configured[64] = {0};
-    using cfg = Cfg<256, true, EPI == EPI_ADDNORM>;
-    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<256, EPI, true>, cfg::SMEM, configured);
+    using cfg = Cfg<BN, true, EPI == EPI_ADDNORM>;
+    cudaError_t e0 = ensure_dynamic_smem(k_gemm_tcgen05<BN, EPI, true>, cfg::SMEM, configured);
     if (e0 != cudaSuccess) return e0;
-    const int tiles = (g.N / 256) * ((g.M + 2 * BM - 1) / (2 * BM));
+    const int tiles = (g.N / BN) * ((g.M + 2 * BM - 1) / (2 * BM));
     const int pairs = num_sms() / 2;
     const int grid = 2 * (tiles < pairs ? tiles : pairs);
-    return launch_kc(k_gemm_tcgen05<256, EPI, true>, dim3(grid), dim3(NUM_THREADS), (size_t)cfg::SMEM, s, 2,
+    return launch_kc(k_gemm_tcgen05<BN, EPI, true>, dim3(grid), dim3(NUM_THREADS), (size_t)cfg::SMEM, s, 2,
                      ma, mw, mc, mh, g);
 }
 
@@ -872,7 +872,8 @@ cudaError_t launch_bn(int bn, const CUtensorMap& ma, const CUtensorMap& mw, cons
         case 32: return launch<32, EPI>(ma, mw, mc, mh, g, s);
         case 64: return launch<64, EPI>(ma, mw, mc, mh, g, s);
         case 128: return launch<128, EPI>(ma, mw, mc, mh, g, s);
-        case 512: return launch_pair<EPI>(ma, mw, mc, mh, g, s);  // 256 x 256 on a CTA pair
+        case 512: return launch_pair<256, EPI>(ma, mw, mc, mh, g, s);  // 256 x 256 on a CTA pair
+        case 640: return launch_pair<128, EPI>(ma, mw, mc, mh, g, s);  // 256 x 128 on a CTA pair
         default: return launch<256, EPI>(ma, mw, mc, mh, g, s);
     }
 }
@@ -889,12 +890,13 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
                  M, N, K);
         return -1;
     }
-    if (force_bn != 0 && force_bn != 32 && force_bn != 64 && force_bn != 128 && force_bn != 256 && force_bn != 512) {
-        snprintf(err, errlen, "gemm: tile %d is not one of 32, 64, 128, 256 (one CTA) or 512 (CTA pair)", force_bn);
+    if (force_bn != 0 && force_bn != 32 && force_bn != 64 && force_bn != 128 && force_bn != 256 && force_bn != 512 &&
+        force_bn != 640) {
+        snprintf(err, errlen, "gemm: tile %d is not one of 32, 64, 128, 256 (one CTA) or 512, 640 (CTA pair)", force_bn);
         return -1;
     }
-    const bool force_pair = force_bn == 512;
-    if (force_pair) force_bn = 256;
+    const bool force_pair = force_bn >= 512;
+    if (force_pair) force_bn = 768 - force_bn;  // 512 -> 256 columns, 640 -> 128
     int bn = force_bn ? force_bn : gemm_tcgen05_tile_n(M, N, K);
     while (bn > max_bn) bn >>= 1;
     if (bn < 32 || N % bn != 0) {
@@ -902,7 +904,10 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
         return -1;
     }
     // large problems: 256 x 256 tiles on CTA pairs (a third less operand traffic per FLOP)
-    const bool pair = bn == 256 && (force_pair || (!force_bn && (long)((M + 255) / 256) * (N / 256) >= num_sms() / 2));
+    // (measured on the decoder's shapes: the pair tile wins from about 0.6 tiles per CTA pair upwards)
+    const long pair_tiles = N % 256 == 0 ? (long)((M + 255) / 256) * (N / 256) : 0;
+    const bool pair = force_pair || (!force_bn && max_bn >= 256 && pair_tiles * 5 >= (long)(num_sms() / 2) * 3);
+    if (pair && !force_pair) bn = 256;
     CUtensorMap ma, mw, mc, mh;
     memset(&mc, 0, sizeof(mc));
     memset(&mh, 0, sizeof(mh));
@@ -915,17 +920,17 @@ int run(int epi, const bf16* A, const bf16* W, GemmArgs& g, int force_bn, int ma
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed for the bf16 output (M=%d N=%d)", M, N);
         return -3;
     }
-    if (!make_map(&ma, A, map_rows, K, BM) || !make_map(&mw, W, N, K, pair ? 128 : bn)) {
+    if (!make_map(&ma, A, map_rows, K, BM) || !make_map(&mw, W, N, K, pair ? bn / 2 : bn)) {
         snprintf(err, errlen, "gemm: cuTensorMapEncodeTiled failed (M=%d N=%d K=%d)", M, N, K);
         return -3;
     }
     cudaError_t e;
     switch (epi) {
-        case EPI_STORE: e = launch_bn<EPI_STORE>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
-        case EPI_ADD: e = launch_bn<EPI_ADD>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
-        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
-        case EPI_ADDNORM: e = launch_bn<EPI_ADDNORM>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
-        default: e = launch_bn<EPI_QKV>(pair ? 512 : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_STORE: e = launch_bn<EPI_STORE>(pair ? 768 - bn : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_ADD: e = launch_bn<EPI_ADD>(pair ? 768 - bn : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_SWIGLU: e = launch_bn<EPI_SWIGLU>(pair ? 768 - bn : bn, ma, mw, mc, mh, g, s); break;
+        case EPI_ADDNORM: e = launch_bn<EPI_ADDNORM>(pair ? 768 - bn : bn, ma, mw, mc, mh, g, s); break;
+        default: e = launch_bn<EPI_QKV>(pair ? 768 - bn : bn, ma, mw, mc, mh, g, s); break;
     }
     if (e != cudaSuccess) {
         snprintf(err, errlen, "gemm launch: %s", cudaGetErrorString(e));
