@@ -32,16 +32,6 @@ def orc_params(w, seed, greedy=False, window=None, history=None, exec_mode=0, ga
                          seed=seed)
 
 
-def bf16_logit_tol(sigma, n_layers):
-    """Max-abs logit tolerance of a bf16 model against the oracle.  Every bf16 rounding point injects a relative
-    error of rms 2^-9 / sqrt(3); a block feeds about three such stages into the residual stream, so after L
-    layers (plus the final norm) the residual carries a relative noise of about (2^-9 / sqrt 3) sqrt(6L + 1),
-    which a logit of scale sigma inherits.  5.5 standard deviations cover the maximum over the ~10^6..10^8 logits
-    compared.  Never tighter than the 2e-2 the task states for unit-scale logits.  (std_estimate, max_tol)."""
-    std = max(sigma, 1e-6) * (2.0 ** -9 / np.sqrt(3.0)) * np.sqrt(6.0 * n_layers + 1.0)
-    return std, max(2e-2, 5.5 * std)
-
-
 def noise_floor(model, w, toks_row, label, c, norm_folded=False):
     """Logit noise floor of bf16 activations at one window: the oracle against ITSELF in its diagnostic form --
     every dot product accumulated in fp32 instead of double, the attention weights rounded to bf16 before they

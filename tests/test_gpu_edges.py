@@ -190,10 +190,13 @@ def test_bf16_model_with_head_size_32_and_unsupported_head_sizes():
     toks, k, lab = synth.make_inputs(w)
     ctx = binding.Context(sh, img, w.batch, w.window)
     model = O.Model(sh, img)
-    rep = G.lockstep(ctx, model, w, toks, k, lab, 3)
-    std, tol = G.bf16_logit_tol(rep["logit_std"], sh.n_layers)
-    assert rep["max_logit_err"] <= tol and rep["abs_err_sum"] / rep["abs_err_n"] <= std
-    assert rep["max_p_err"] <= 1e-6 and rep["replay_mismatch"] == 0
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 3, floor_every_round=True)
+    # logits against the noise floor measured on the same windows (the context folds its RMSNorm: factor 1.5 on the
+    # mean, measured 1.25; the maximum over these few thousand logits measured 1.43 x the floor's)
+    G.check_logits_against_floor(rep, rep["floor_max"], rep["floor_sum"] / rep["floor_n"], "head size 32",
+                                 max_factor=1.8, mean_factor=1.5)
+    assert rep["max_p_err"] <= 1e-6
+    G.check_flips_explained(rep)
     assert rep["same"] >= 0.9 * rep["tokens"]
     ctx.hbsjd_destroy()
     bad = synth.ModelShape(1, 256, 2, 256, 512, 4, 4, 5, "bf16")         # dh = 128
