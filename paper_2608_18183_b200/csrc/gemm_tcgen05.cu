@@ -552,11 +552,6 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                     float4 hcur[8];
 #pragma unroll
                     for (int v = 0; v < 8; ++v) hcur[v] = hbuf[u][v];
-                    if (c0 + 96 < BN && row < M) {  // the chunk three ahead takes the slot this chunk frees next
-                        const float4* hp = reinterpret_cast<const float4*>(g.C + (size_t)row * N + col + 96);
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) hbuf[(u + 3) % UNR][v] = hp[v];
-                    }
                     // new residual = old + acc (one fp32 addition per element, as the reduce-add form did)
                     float ss = 0.f;
 #pragma unroll
@@ -609,6 +604,14 @@ __global__ void __launch_bounds__(NUM_THREADS) k_gemm_tcgen05(const __grid_const
                                      "r"(col), "r"(m0 + quarter * 32), "r"(sb16)
                                      : "memory");
                         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    }
+                    // The chunk three ahead takes the register slot this chunk has freed.  Requested only now, behind
+                    // the proxy fence above: a fence waits for the loads its thread has in flight, so a request in
+                    // front of it would cost the fence a full memory latency per chunk.
+                    if (c0 + 96 < BN && row < M) {
+                        const float4* hp = reinterpret_cast<const float4*>(g.C + (size_t)row * N + col + 96);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) hbuf[(u + 3) % UNR][v] = hp[v];
                     }
                     continue;
                 }
