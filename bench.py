@@ -301,7 +301,10 @@ def main():
         name: {"launches": b["launches"], "ms_per_step": b["ms"] / args.steps,
                "achieved": b["work"] / (b["ms"] * 1e-3) / 1e12 if b["ms"] > 0 else 0.0,
                "frac": b["work"] / (b["ms"] * 1e-3) / 1e12 / pk["bf16_tflops_sustained"] if b["ms"] > 0 else 0.0,
-               "frac_net_of_launch_floor": net(b) / 1e12 / pk["bf16_tflops_sustained"]}
+               "frac_net_of_launch_floor": net(b) / 1e12 / pk["bf16_tflops_sustained"],
+               # the same launches against the HBM roofline (operands read once, outputs written): the bound that
+               # matters where the rows are few and a launch streams its weight matrix
+               "hbm_frac": b["bytes"] / (b["ms"] * 1e-3) / 1e9 / pk["hbm_gbs"] if b["ms"] > 0 else 0.0}
         for name, b in prof["gemm_by_rows"].items()}
     if w.shape.dtype != "bf16":
         roof.update(bound="alu", peak=72.0, peak_source="fp32 CUDA-core FMA: 148 SMs x 128 lanes x 2 x 1.9 GHz")

@@ -322,6 +322,7 @@ typedef struct {
     double gemm_ms_by_rows[4];
     double gemm_work_by_rows[4];
     int64_t gemm_launches_by_rows[4];
+    double gemm_bytes_by_rows[4];   /* algorithmic bytes: operands read once, outputs written (residual: read + written) */
 } hbsjd_kernel_profile;
 int hbsjd_profile(hbsjd_ctx *c, int enable);
 int hbsjd_profile_read(hbsjd_ctx *c, hbsjd_kernel_profile *out);

@@ -48,7 +48,7 @@ class hbsjd_stats(C.Structure):
 class hbsjd_kernel_profile(C.Structure):
     _fields_ = [("ms", C.c_double * 4), ("work", C.c_double * 4), ("launches", C.c_int64 * 4),
                 ("dropped", C.c_int64), ("gemm_ms_by_rows", C.c_double * 4), ("gemm_work_by_rows", C.c_double * 4),
-                ("gemm_launches_by_rows", C.c_int64 * 4)]
+                ("gemm_launches_by_rows", C.c_int64 * 4), ("gemm_bytes_by_rows", C.c_double * 4)]
 
 
 PROF_CLASSES = ("gemm", "attention", "accept", "other")
@@ -205,7 +205,8 @@ class Context:
         return {n: dict(ms=p.ms[i], work=p.work[i], launches=p.launches[i]) for i, n in enumerate(PROF_CLASSES)} | {
             "dropped": p.dropped,
             "gemm_by_rows": {n: dict(ms=p.gemm_ms_by_rows[i], work=p.gemm_work_by_rows[i],
-                                     launches=p.gemm_launches_by_rows[i]) for i, n in enumerate(PROF_GEMM_ROW_BINS)}}
+                                     launches=p.gemm_launches_by_rows[i], bytes=p.gemm_bytes_by_rows[i])
+                             for i, n in enumerate(PROF_GEMM_ROW_BINS)}}
 
     def hbsjd_profile_launch_floor(self, reps=200) -> float:
         """Median event bracket of an empty kernel launch, microseconds."""

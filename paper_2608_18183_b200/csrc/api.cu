@@ -65,7 +65,7 @@ struct hbsjd_ctx {
     int32_t* m_sync;                              // [1] smallest commit of the round (batch-synchronous progress)
     // per-class event timing
     bool profiling;
-    struct ProfSlot { cudaEvent_t a, b; int cls; double work; int rows; };
+    struct ProfSlot { cudaEvent_t a, b; int cls; double work; int rows; double bytes; };
     std::vector<ProfSlot> pool;
     int pool_used;
     int pending_attn;  // attention launches of the current forward whose byte count waits for the counters
@@ -87,7 +87,7 @@ namespace {
 size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 // Brackets the launches issued between prof_begin and prof_end with an event pair of class `cls`.
-int prof_begin(hbsjd_ctx* c, int cls, double work, int rows = 0) {
+int prof_begin(hbsjd_ctx* c, int cls, double work, int rows = 0, double bytes = 0.0) {
     if (!c->profiling) return -1;
     if (c->pool_used >= (int)c->pool.size()) {
         c->prof.dropped++;
@@ -97,6 +97,7 @@ int prof_begin(hbsjd_ctx* c, int cls, double work, int rows = 0) {
     s.cls = cls;
     s.work = work;
     s.rows = rows;
+    s.bytes = bytes;
     cudaEventRecord(s.a, c->stream);
     return c->pool_used++;
 }
@@ -120,6 +121,7 @@ void prof_resolve(hbsjd_ctx* c, double attn_bytes, double accept_bytes) {
             const int bin = s.rows <= 512 ? 0 : s.rows <= 2048 ? 1 : s.rows <= 6144 ? 2 : 3;
             c->prof.gemm_ms_by_rows[bin] += ms;
             c->prof.gemm_work_by_rows[bin] += work;
+            c->prof.gemm_bytes_by_rows[bin] += s.bytes;
             c->prof.gemm_launches_by_rows[bin] += 1;
         }
     }
@@ -155,7 +157,8 @@ int gemm(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int
 template <>
 int gemm<float>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate, int, int,
                 unsigned int, int) {
-    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K, M);
+    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K, M,
+                              4.0 * ((double)M * K + (double)N * K) + 4.0 * M * N * (accumulate ? 2 : 1));
     launch_gemm_simt<float>((const float*)A, (const float*)W, C, M, N, K, accumulate, c->stream);
     prof_end(c, ps);
     c->launches++;
@@ -166,7 +169,8 @@ template <>
 int gemm<bf16>(hbsjd_ctx* c, const void* A, const void* W, float* C, int M, int N, int K, int accumulate,
                int m_cap, int w_constant, unsigned int acc_wait_ns, int tile) {
     c->launches++;
-    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K, M);
+    const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * N * K, M,
+                              2.0 * ((double)M * K + (double)N * K) + 4.0 * M * N * (accumulate ? 2 : 1));
     const int rc = gemm_tcgen05_run((const bf16*)A, (const bf16*)W, C, M, N, K, accumulate, tile, m_cap,
                                     c->st.counters + CNT_ERROR, c->stream, c->err, sizeof(c->err), w_constant,
                                     acc_wait_ns);
@@ -249,6 +253,7 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
     cudaStream_t s = c->stream;
     const KvView kv = kv_view(c);
     const bool fold = c->fold_norm;
+    const double es = 2.0;  // bytes of a bf16 operand / output element (algorithmic byte counts of the profile)
     bf16* a = (bf16*)c->a;  // folded: bf16 copy of the residual stream; separate: the normed operand
     const NormIn nin = {fold ? c->ssq : nullptr, c->d.rms_eps};
     int32_t* eflag = c->st.counters + CNT_ERROR;
@@ -261,7 +266,9 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
     };
     // residual update h += A W^T
     auto residual = [&](const void* A, const void* W, int K) {
-        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * D * K, M);
+        // operands, the fp32 residual read and written, and (folded norm) its bf16 copy
+        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * D * K, M,
+                                  es * ((double)M * K + (double)D * K) + 8.0 * M * D + (fold ? 2.0 * M * D : 0.0));
         int rc;
         if (fold)
             rc = gemm_tcgen05_addnorm((const bf16*)A, (const bf16*)W, c->h, a, c->ssq, M, D, K, Mcap, eflag, s, c->err,
@@ -280,7 +287,8 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
         const LayerW& w = c->layers[l];
         int rc, ps;
         if (!fold) norm(w.g_attn);
-        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D, M);
+        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 3 * D * D, M,
+                        es * ((double)M * D + 3.0 * D * D) + es * 3.0 * M * D);  // q, k, v written
         rc = gemm_tcgen05_qkv(a, (const bf16*)w.w_qkv, (bf16*)c->q, st, S, l, c->rope_cs, kv, Mcap, nin, eflag, s,
                               c->err, sizeof(c->err));
         prof_end(c, ps);
@@ -298,7 +306,8 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
         if ((rc = residual(c->o, w.w_o, D))) return done(rc);
         if (l == stop_layer && stop_stage == 0) return 0;
         if (!fold) norm(w.g_ffn);
-        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D, M);
+        ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * 2 * F * D, M,
+                        es * ((double)M * D + 2.0 * F * D) + es * (double)M * F);
         rc = gemm_tcgen05_swiglu(a, (const bf16*)w.w_13, (bf16*)c->act, M, 2 * F, D, Mcap, nin, eflag, s, c->err,
                                  sizeof(c->err));
         prof_end(c, ps);
@@ -309,7 +318,8 @@ int forward<bf16>(hbsjd_ctx* c, int S, bool want_logits, int stop_layer, int sto
     }
     if (want_logits) {
         if (!fold) norm(c->g_out);
-        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * st.V * D, M);
+        const int ps = prof_begin(c, HBSJD_PROF_GEMM, 2.0 * M * st.V * D, M,
+                                  es * ((double)M * D + (double)st.V * D) + 4.0 * M * st.V);
         const int rc = gemm_tcgen05_head(a, (const bf16*)c->w_head, c->logits, M, st.V, D, Mcap, nin, eflag, s,
                                          c->err, sizeof(c->err));
         prof_end(c, ps);
