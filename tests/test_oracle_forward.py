@@ -118,6 +118,44 @@ def test_noise_floor_of_bf16_activations_at_full_depth():
     assert np.array_equal(a, b)
 
 
+def test_diagnostic_switches_are_what_they_say(tiny):
+    """The three diagnostic switches of the oracle (they only serve the noise-floor measurements of the GPU tests)
+    pinned one by one on a model WITHOUT bf16 rounding, where their effect is known in closed form: the folded
+    RMSNorm is the same mathematics (gain into the weight row, row factor after the product), so with random
+    gains it must agree to double rounding; fp32 sums differ at fp32 resolution and no more; bf16 attention
+    weights differ at bf16 resolution of a probability and no more.  And with everything switched off again the
+    oracle proper is back, bit for bit."""
+    w, img = tiny
+    img = img.copy()
+    table, _ = synth.tensor_table(w.shape)
+    rng = np.random.default_rng(5)
+    for name, r, c, off in table:  # random gains, so that a fold that loses or misplaces the gain shows
+        if name.split(".")[-1] in ("g_attn", "g_ffn") or name == "g_out":
+            img[off:off + 4 * c] = np.frombuffer((0.5 + rng.random(c)).astype(np.float32).tobytes(), dtype=np.uint8)
+    m = O.Model(w.shape, img, act_bf16=False)
+    seq = _seq(w.shape, 40, 3)
+    ref = m.forward_full(2, seq).astype(np.float64)
+    scale = float(ref.std())
+
+    def with_diag(**kw):
+        m.set_diag(**kw)
+        try:
+            return m.forward_full(2, seq).astype(np.float64)
+        finally:
+            m.set_diag()
+
+    d_fold = np.abs(with_diag(norm_folded=True) - ref).max()
+    d_f32 = np.abs(with_diag(acc_f32=True) - ref).max()
+    d_att = np.abs(with_diag(attn_w_bf16=True) - ref).max()
+    assert d_fold < 2e-6 * scale, d_fold                  # the outputs are stored as fp32: same to their last bit or two
+    assert 1e-8 * scale < d_f32 < 1e-4 * scale, d_f32     # fp32 sums over <= 192 terms
+    assert 1e-5 * scale < d_att < 3e-2 * scale, d_att     # 2^-9 relative on the attention weights
+    assert np.array_equal(m.forward_full(2, seq).astype(np.float64), ref)
+    # a fold that dropped the gain would not pass: unit gains move the logits by far more than any of the above
+    unit = O.Model(w.shape, tiny[1], act_bf16=False).forward_full(2, seq)
+    assert np.abs(unit - ref).max() > 1e-2 * scale
+
+
 def test_cached_window_forward_equals_full_recompute(tiny):
     w, img = tiny
     m = O.Model(w.shape, img)
