@@ -92,3 +92,19 @@ def test_fullsize_one_image_to_completion(big):
     rep = G.lockstep(ctx, model, w, toks, k2, lab, 29, image_ids=[b], park_others=False)
     assert rep["tokens"] == 40
     _check_against_floor(ctx, rep, model, w, toks, lab, k2, [b], f"{w.name} image {b} to completion")
+
+
+def test_fullsize_greedy_verification_in_lockstep(big):
+    """Greedy verification (Eq. 4) at full vocabulary and batch: two images of workload B followed for four rounds;
+    an argmax that differs from the oracle's must be a near-tie of the oracle's own logits, which the per-flip
+    replay establishes (the oracle's verification fed the GPU's probabilities reproduces the GPU's decision)."""
+    w, weights, ctx, toks, k, lab = big
+    if w.name != "B":
+        pytest.skip("one configuration is enough for the greedy rule at full size")
+    order = np.argsort(k, kind="stable")
+    ids = sorted({int(order[0]), int(order[-1])})
+    model = O.Model(w.shape, weights)
+    rep = G.lockstep(ctx, model, w, toks, k, lab, 31, greedy=True, image_ids=ids, max_rounds=4, park_others=False)
+    assert rep["tokens"] >= 4 * len(ids)
+    _check_against_floor(ctx, rep, model, w, toks, lab, k, ids, f"{w.name} greedy ids {ids}")
+
