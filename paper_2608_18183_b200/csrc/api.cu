@@ -990,7 +990,7 @@ int hbsjd_profile(hbsjd_ctx* c, int enable) {
     CK(cudaStreamSynchronize(c->stream));
     c->profiling = enable != 0;
     c->pool_used = 0;
-    memset(&c->prof, 0, sizeof(c->prof));
+    if (enable) memset(&c->prof, 0, sizeof(c->prof));  // switching off keeps the totals readable
     return HBSJD_OK;
 }
 

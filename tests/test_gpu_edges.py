@@ -226,3 +226,27 @@ def test_images_do_not_depend_on_their_batch_mates():
         for b in keep:
             np.testing.assert_array_equal(out[b], ref[b])
     ctx.hbsjd_destroy()
+
+
+def test_kernel_profile_bins_add_up():
+    """Per-class event timing: the GEMM class split by activation rows adds up to the class, every bin that has
+    launches has time, FLOPs and algorithmic bytes, and switching the profile off stops the accounting."""
+    w = synth.WORKLOADS["small_bf16"]
+    toks, k, lab = synth.make_inputs(w)
+    ctx = binding.Context(w.shape, G.weights_for(w), w.batch, w.window)
+    ctx.hbsjd_profile(True)
+    _, st = ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 3))
+    p = ctx.hbsjd_profile_read()
+    ctx.hbsjd_profile(False)
+    g, bins = p["gemm"], p["gemm_by_rows"]
+    assert g["launches"] > 0 and p["attention"]["launches"] > 0 and p["accept"]["launches"] == st["rounds"]
+    assert sum(b["launches"] for b in bins.values()) == g["launches"]
+    assert abs(sum(b["ms"] for b in bins.values()) - g["ms"]) <= 1e-6 * g["ms"]
+    assert abs(sum(b["work"] for b in bins.values()) - g["work"]) <= 1e-9 * g["work"]
+    for b in bins.values():
+        assert (b["launches"] > 0) == (b["ms"] > 0) == (b["work"] > 0) == (b["bytes"] > 0)
+    assert bins["rows>6144"]["launches"] == 0                  # this context has at most 2 x batch x window rows
+    ctx.hbsjd_rollout(G.dev(toks), G.dev(k), G.dev(lab), G.gpu_params(w, 3))
+    assert ctx.hbsjd_profile_read()["gemm"]["launches"] == g["launches"]
+    ctx.hbsjd_destroy()
+
